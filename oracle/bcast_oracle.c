@@ -1,0 +1,315 @@
+/*
+ * bcast_oracle.c -- TEST INFRASTRUCTURE, NOT PART OF THE PRODUCT.
+ *
+ * A plain, slow, single-threaded CPU simulation of the scatter-ring-allgather
+ * broadcast over P simulated processes, each with its own host buffer, written
+ * from the paper "A Bandwidth-saving Optimization for MPI Broadcast Collective
+ * Operation" (Zhou, Marjanovic, Niethammer, Gracia).  It exists so that tests,
+ * the smoke check and the CPU-baseline leg of the benchmark have something to
+ * compare the CUDA library against.  It shares no code, header or table with
+ * that library, and nothing in the library may call it.
+ *
+ * What it follows:
+ *   - Section III-A (Figs. 1-2):  binomial scatter, the root's message cut into
+ *     P chunks of scatter_size = ceil(nbytes / P) bytes.
+ *   - Section III-A (Fig. 3):     native "enclosed" ring allgather, P-1 steps,
+ *     every process sends and receives in every step.
+ *   - Section IV (Figs. 4-5 and the pseudo-code listing): tuned "non-enclosed"
+ *     ring allgather; each process computes (step, flag) and turns send-only or
+ *     receive-only once  step > P - i.
+ *
+ * Every simulated process runs the per-process logic of the listing; a message
+ * is the pair of one process's send and its right neighbour's receive, and the
+ * simulation checks that they match before it copies anything.  No blocking,
+ * fusion or reordering: one memcpy per message, steps in the paper's order.
+ *
+ * Readings taken where the paper is silent (each also listed in the design
+ * notes of the repository):
+ *   - nbytes = count * length of the listing's signature.
+ *   - the opaque binomial_tree() call is the tree of Figs. 1-2: in level t
+ *     (mask m = 2^(L-1-t), L = ceil(log2 P)) every relative rank r that is a
+ *     multiple of 2m and has r + m < P sends the chunks [r+m, min(r+2m, P))
+ *     to relative rank r + m.
+ *   - chunk indices and displacements are RELATIVE to the root (the listing
+ *     displaces by the relative rank); src/dst ranks are absolute.
+ *   - zero-length messages (chunks past the end of a short message) are still
+ *     messages: the listing clamps the count to 0 and still makes the call.
+ *     Their offset is reported clipped to nbytes.
+ *   - inside one step, messages are listed by ascending destination rank.
+ *   - a "message transfer" in the paper's 56/44 and 90/75 counts is a ring
+ *     message; scatter messages are counted separately.
+ *
+ * Pinned by tests/test_oracle_pins.py against the worked examples of
+ * Figs. 1-5, the printed message counts, closed forms, MPI broadcast
+ * semantics and a brute-force ownership enumeration.  Nothing is unpinned.
+ */
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+enum { ORC_OK = 0, ORC_E_ARG = -1, ORC_E_NOMEM = -2, ORC_E_CAP = -3,
+       ORC_E_NOT_HELD = -4,      /* a sender did not hold what it sends          */
+       ORC_E_UNMATCHED = -5,     /* a send without the matching receive          */
+       ORC_E_STEPFLAG = -6,      /* (step, flag) left undefined by the loop      */
+       ORC_E_OVERLAP = -7,       /* a step reads a range that the step writes    */
+       ORC_E_INCOMPLETE = -8,    /* some process misses a chunk at the end       */
+       ORC_E_MISMATCH = -9 };    /* some buffer differs from the root's message  */
+
+/* schedule record: 9 x int64, in this order */
+enum { F_PHASE = 0, F_STEP, F_SRC, F_DST, F_CHUNK, F_NCHUNKS, F_OFFSET, F_LEN, F_DEP, F_NFIELDS };
+enum { PH_SCATTER = 0, PH_RING = 1 };
+enum { SEND_ONLY = 0, RECV_ONLY = 1, FLAG_UNSET = -1 };
+
+typedef struct {
+    int P, root;
+    uint64_t n, S;
+    uint8_t *const *buf;          /* NULL: schedule and counters only */
+    int64_t *sched, cap, len;
+    uint64_t *bytes_sent, *bytes_recv, *msgs_sent, *msgs_recv;   /* [2][P] */
+    uint8_t *holds;               /* holds[k*P + c]: process k (absolute) holds chunk c (relative) */
+    int *rd_lo, *rd_hi;           /* per process: chunk range read from it in the current step */
+    int64_t *writer;              /* writer[k*P + c]: schedule index of the message that last wrote it, -1 = never */
+} sim_t;
+
+static uint64_t umin(uint64_t a, uint64_t b) { return a < b ? a : b; }
+
+/* first byte of relative chunk c, clipped to the message (Section IV listing: disp = rel * scatter_size) */
+static uint64_t chunk_begin(const sim_t *s, int c) { return umin((uint64_t)c * s->S, s->n); }
+
+/* length of relative chunk c: min(scatter_size, nbytes - c*scatter_size), clamped at 0 (listing) */
+static uint64_t chunk_len(const sim_t *s, int c)
+{
+    uint64_t b = (uint64_t)c * s->S;
+    if (b >= s->n) return 0;
+    return umin(s->S, s->n - b);
+}
+
+static int rel_of(const sim_t *s, int k) { return k >= s->root ? k - s->root : k - s->root + s->P; }
+static int abs_of(const sim_t *s, int r) { return (r + s->root) % s->P; }
+
+typedef struct { int src, dst, chunk, nchunks; } pending_t;
+
+static int by_dst(const void *a, const void *b)
+{
+    return ((const pending_t *)a)->dst - ((const pending_t *)b)->dst;
+}
+
+/* Deliver the messages of one step: check, record, count, copy. */
+static int deliver_step(sim_t *s, int phase, int step, pending_t *m, int nm)
+{
+    const int P = s->P;
+    qsort(m, (size_t)nm, sizeof *m, by_dst);
+
+    /* a process can only send what has arrived at it in an earlier step */
+    for (int a = 0; a < nm; a++)
+        for (int c = m[a].chunk; c < m[a].chunk + m[a].nchunks; c++)
+            if (!s->holds[(size_t)m[a].src * P + c]) return ORC_E_NOT_HELD;
+    /* all sends of a step see the buffers as they were when the step began: nothing a message
+       of this step writes may be read by a message of this step, so that copying the messages
+       one after the other equals copying them at once */
+    for (int k = 0; k < P; k++) s->rd_lo[k] = s->rd_hi[k] = 0;      /* chunk range read from process k */
+    for (int a = 0; a < nm; a++) {
+        if (s->rd_hi[m[a].src] != s->rd_lo[m[a].src]) return ORC_E_UNMATCHED;   /* one send per process and step */
+        s->rd_lo[m[a].src] = m[a].chunk; s->rd_hi[m[a].src] = m[a].chunk + m[a].nchunks;
+    }
+    for (int a = 0; a < nm; a++)
+        if (m[a].chunk < s->rd_hi[m[a].dst] && s->rd_lo[m[a].dst] < m[a].chunk + m[a].nchunks)
+            return ORC_E_OVERLAP;
+
+    for (int a = 0; a < nm; a++) {
+        const int c0 = m[a].chunk, c1 = c0 + m[a].nchunks;
+        const uint64_t off = chunk_begin(s, c0);
+        uint64_t len = 0;
+        for (int c = c0; c < c1; c++) len += chunk_len(s, c);
+        if (s->len + a >= s->cap) return ORC_E_CAP;
+        int64_t *rec = s->sched + (s->len + a) * F_NFIELDS;
+        rec[F_PHASE] = phase;  rec[F_STEP] = step;
+        rec[F_SRC] = m[a].src; rec[F_DST] = m[a].dst;
+        rec[F_CHUNK] = c0;     rec[F_NCHUNKS] = m[a].nchunks;
+        rec[F_OFFSET] = (int64_t)off; rec[F_LEN] = (int64_t)len;
+        rec[F_DEP] = s->writer[(size_t)m[a].src * P + c0];
+
+        s->bytes_sent[(size_t)phase * P + m[a].src] += len;
+        s->bytes_recv[(size_t)phase * P + m[a].dst] += len;
+        s->msgs_sent[(size_t)phase * P + m[a].src] += 1;
+        s->msgs_recv[(size_t)phase * P + m[a].dst] += 1;
+
+        if (s->buf && len) memcpy(s->buf[m[a].dst] + off, s->buf[m[a].src] + off, (size_t)len);
+    }
+    /* ownership changes only after every message of the step has been read */
+    for (int a = 0; a < nm; a++) {
+        /* records of this step were appended in the same order as m[] */
+        const int64_t idx = s->len + a;
+        for (int c = m[a].chunk; c < m[a].chunk + m[a].nchunks; c++) {
+            s->holds[(size_t)m[a].dst * P + c] = 1;
+            s->writer[(size_t)m[a].dst * P + c] = idx;
+        }
+    }
+    s->len += nm;
+    return ORC_OK;
+}
+
+/* Section III-A, Figs. 1-2: binomial scatter from relative rank 0. */
+static int scatter_phase(sim_t *s, int L, pending_t *m)
+{
+    const int P = s->P;
+    for (int t = 0; t < L; t++) {
+        const int mask = 1 << (L - 1 - t);
+        int nm = 0;
+        for (int r = 0; r < P; r += 2 * mask) {          /* roots of the sub-trees alive at this level */
+            if (r + mask >= P) continue;                 /* no process there (non-power-of-two P)   */
+            const int hi = (r + 2 * mask < P) ? r + 2 * mask : P;
+            m[nm].src = abs_of(s, r);
+            m[nm].dst = abs_of(s, r + mask);
+            m[nm].chunk = r + mask;                      /* the child gets its own chunk ...         */
+            m[nm].nchunks = hi - (r + mask);             /* ... and those of all its descendants     */
+            nm++;
+        }
+        int rc = deliver_step(s, PH_SCATTER, t, m, nm);
+        if (rc) return rc;
+    }
+    return ORC_OK;
+}
+
+/* Section IV, "added code" of the listing: after how many held chunks a process leaves the
+   two-sided exchange (step), and whether it then only sends or only receives (flag). */
+static void step_and_flag(int P, int r, int *step, int *flag)
+{
+    int mask = 1;
+    while (mask < P) mask <<= 1;                         /* 2^ceil(log2 P) */
+    *step = 0; *flag = FLAG_UNSET;
+    for (; mask > 1; mask >>= 1) {
+        const int rr = (r + 1 < P) ? r + 1 : r + 1 - P;  /* right neighbour, relative */
+        if (rr % mask == 0) {                            /* the right neighbour roots a sub-tree   */
+            *step = (rr + mask > P) ? P - rr : mask;     /* of this many chunks: it stops taking   */
+            *flag = RECV_ONLY;                           /* them, so this process stops sending    */
+            return;
+        }
+        if (r % mask == 0) {                             /* this process roots a sub-tree: it      */
+            *step = (r + mask > P) ? P - r : mask;       /* stops receiving and only sends         */
+            *flag = SEND_ONLY;
+            return;
+        }
+    }
+}
+
+/* Section III-A Fig. 3 (native) and Section IV Figs. 4-5 + listing (tuned): P-1 ring steps. */
+static int ring_phase(sim_t *s, int tuned, pending_t *m)
+{
+    const int P = s->P;
+    int rc = ORC_OK;
+    int *j = malloc(sizeof(int) * (size_t)P), *jnext = malloc(sizeof(int) * (size_t)P);
+    int *step = malloc(sizeof(int) * (size_t)P), *flag = malloc(sizeof(int) * (size_t)P);
+    uint8_t *sends = malloc((size_t)P), *recvs = malloc((size_t)P);
+    if (!j || !jnext || !step || !flag || !sends || !recvs) { rc = ORC_E_NOMEM; goto out; }
+
+    for (int k = 0; k < P; k++) {
+        j[k] = k;                                        /* first the own chunk goes right ...     */
+        jnext[k] = (P + k - 1) % P;                      /* ... and the left neighbour's comes in  */
+        step_and_flag(P, rel_of(s, k), &step[k], &flag[k]);
+        /* P = 1: the mask loop never runs and there is no ring step that would use the result */
+        if (tuned && P > 1 && flag[k] == FLAG_UNSET) { rc = ORC_E_STEPFLAG; goto out; }
+    }
+
+    for (int i = 1; i < P; i++) {
+        /* what every process does in step i */
+        for (int k = 0; k < P; k++) {
+            if (!tuned || step[k] <= P - i) { sends[k] = 1; recvs[k] = 1; }      /* Sendrecv */
+            else if (flag[k] == RECV_ONLY)  { sends[k] = 0; recvs[k] = 1; }      /* Recv     */
+            else                            { sends[k] = 1; recvs[k] = 0; }      /* Send     */
+        }
+        /* pair each send with the right neighbour's receive */
+        int nm = 0;
+        for (int k = 0; k < P; k++) {
+            const int right = (k + 1) % P;
+            if (sends[k] != recvs[right]) { rc = ORC_E_UNMATCHED; goto out; }
+            if (!sends[k]) continue;
+            const int rel_j = rel_of(s, j[k]);               /* chunk the sender puts on the wire   */
+            const int rel_jnext = rel_of(s, jnext[right]);   /* chunk the receiver expects          */
+            if (rel_j != rel_jnext) { rc = ORC_E_UNMATCHED; goto out; }
+            m[nm].src = k; m[nm].dst = right; m[nm].chunk = rel_j; m[nm].nchunks = 1;
+            nm++;
+        }
+        rc = deliver_step(s, PH_RING, i - 1, m, nm);
+        if (rc) goto out;
+        for (int k = 0; k < P; k++) { j[k] = jnext[k]; jnext[k] = (P + jnext[k] - 1) % P; }
+    }
+out:
+    free(j); free(jnext); free(step); free(flag); free(sends); free(recvs);
+    return rc;
+}
+
+/*
+ * Simulate one broadcast.
+ *   P, root, nbytes   communicator size, root rank, message bytes
+ *   tuned             0: native ring (Section III-A), 1: tuned ring (Section IV)
+ *   buf               P host buffers of nbytes each; buf[root] holds the message.  NULL: no data is
+ *                     moved, only the schedule and the counters are produced.
+ *   sched, cap        room for cap records of 9 int64 (phase, step, src, dst, chunk, nchunks,
+ *                     offset, len, dep); *nsched receives the number written
+ *   bytes_sent ...    four arrays [2][P] (phase, absolute rank), zeroed here
+ * Returns ORC_OK or a negative ORC_E_* code.
+ */
+int oracle_bcast_simulate(int P, int root, uint64_t nbytes, int tuned, uint8_t *const *buf,
+                          int64_t *sched, int64_t cap, int64_t *nsched,
+                          uint64_t *bytes_sent, uint64_t *bytes_recv,
+                          uint64_t *msgs_sent, uint64_t *msgs_recv)
+{
+    if (P < 1 || root < 0 || root >= P || !sched || !nsched || cap < 0 ||
+        !bytes_sent || !bytes_recv || !msgs_sent || !msgs_recv)
+        return ORC_E_ARG;
+
+    sim_t s;
+    memset(&s, 0, sizeof s);
+    s.P = P; s.root = root; s.n = nbytes;
+    s.S = (nbytes + (uint64_t)P - 1) / (uint64_t)P;          /* scatter_size, Section IV listing */
+    s.buf = buf; s.sched = sched; s.cap = cap; s.len = 0;
+    s.bytes_sent = bytes_sent; s.bytes_recv = bytes_recv; s.msgs_sent = msgs_sent; s.msgs_recv = msgs_recv;
+    memset(bytes_sent, 0, sizeof(uint64_t) * 2 * (size_t)P);
+    memset(bytes_recv, 0, sizeof(uint64_t) * 2 * (size_t)P);
+    memset(msgs_sent, 0, sizeof(uint64_t) * 2 * (size_t)P);
+    memset(msgs_recv, 0, sizeof(uint64_t) * 2 * (size_t)P);
+
+    int rc = ORC_OK;
+    pending_t *m = malloc(sizeof(pending_t) * (size_t)P);
+    s.holds = calloc((size_t)P * (size_t)P, 1);
+    s.writer = malloc(sizeof(int64_t) * (size_t)P * (size_t)P);
+    s.rd_lo = malloc(sizeof(int) * (size_t)P);
+    s.rd_hi = malloc(sizeof(int) * (size_t)P);
+    if (!m || !s.holds || !s.writer || !s.rd_lo || !s.rd_hi) { rc = ORC_E_NOMEM; goto out; }
+    for (size_t x = 0; x < (size_t)P * (size_t)P; x++) s.writer[x] = -1;
+    for (int c = 0; c < P; c++) s.holds[(size_t)root * P + c] = 1;   /* the root has the whole message */
+
+    int L = 0;
+    while ((1 << L) < P) L++;                                 /* ceil(log2 P) scatter levels */
+
+    rc = scatter_phase(&s, L, m);
+    if (rc) goto out;
+    rc = ring_phase(&s, tuned, m);
+    if (rc) goto out;
+
+    /* MPI broadcast semantics (Section III-A): on return every process has the root's message */
+    for (size_t x = 0; x < (size_t)P * (size_t)P; x++)
+        if (!s.holds[x]) { rc = ORC_E_INCOMPLETE; goto out; }
+    if (buf && nbytes)
+        for (int k = 0; k < P; k++)
+            if (memcmp(buf[k], buf[root], (size_t)nbytes) != 0) { rc = ORC_E_MISMATCH; goto out; }
+out:
+    *nsched = s.len;
+    free(m); free(s.holds); free(s.writer); free(s.rd_lo); free(s.rd_hi);
+    return rc;
+}
+
+/* scatter_size for the caller's convenience (Section IV listing) */
+uint64_t oracle_bcast_scatter_size(int P, uint64_t nbytes)
+{
+    return P < 1 ? 0 : (nbytes + (uint64_t)P - 1) / (uint64_t)P;
+}
+
+/* (step, flag) of one relative rank, exposed so that tests can pin it on its own */
+int oracle_bcast_step_flag(int P, int rel_rank, int *step, int *flag)
+{
+    if (P < 1 || rel_rank < 0 || rel_rank >= P || !step || !flag) return ORC_E_ARG;
+    step_and_flag(P, rel_rank, step, flag);
+    return ORC_OK;
+}

@@ -1,0 +1,155 @@
+"""ctypes front end of the CPU oracle (oracle/bcast_oracle.c).
+
+TEST INFRASTRUCTURE, NOT PART OF THE PRODUCT: only the tests, the smoke check and the
+CPU-baseline / reference legs of the benchmark may import this module.  It imports nothing
+from the CUDA package and the CUDA package imports nothing from here.
+
+The C file is compiled with gcc on first use into ``oracle/_build``.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+import time
+from dataclasses import dataclass
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "bcast_oracle.c")
+_LIB = os.path.join(_HERE, "_build", "libbcast_oracle.so")
+
+NATIVE, TUNED = 0, 1
+SCATTER, RING = 0, 1
+SEND_ONLY, RECV_ONLY = 0, 1
+
+#: column names of the schedule array returned by :func:`simulate`
+FIELDS = ("phase", "step", "src", "dst", "chunk", "nchunks", "offset", "len", "dep")
+
+ERRORS = {
+    -1: "bad argument", -2: "out of memory", -3: "schedule capacity exceeded",
+    -4: "a sender did not hold what it sends", -5: "send without matching receive",
+    -6: "(step, flag) undefined", -7: "a step reads what it writes",
+    -8: "a process misses a chunk at the end", -9: "a buffer differs from the root's message",
+}
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc if the shared object is missing or older than the source."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        os.makedirs(os.path.dirname(_LIB), exist_ok=True)
+        tmp = _LIB + f".{os.getpid()}.tmp"
+        subprocess.check_call(["gcc", "-O2", "-Wall", "-Wextra", "-shared", "-fPIC", "-o", tmp, _SRC])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+_lib = None
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        u64p = ctypes.POINTER(ctypes.c_uint64)
+        lib.oracle_bcast_simulate.restype = ctypes.c_int
+        lib.oracle_bcast_simulate.argtypes = [
+            ctypes.c_int, ctypes.c_int, ctypes.c_uint64, ctypes.c_int, ctypes.POINTER(ctypes.c_void_p),
+            ctypes.POINTER(ctypes.c_int64), ctypes.c_int64, ctypes.POINTER(ctypes.c_int64),
+            u64p, u64p, u64p, u64p]
+        lib.oracle_bcast_scatter_size.restype = ctypes.c_uint64
+        lib.oracle_bcast_scatter_size.argtypes = [ctypes.c_int, ctypes.c_uint64]
+        lib.oracle_bcast_step_flag.restype = ctypes.c_int
+        lib.oracle_bcast_step_flag.argtypes = [ctypes.c_int, ctypes.c_int,
+                                               ctypes.POINTER(ctypes.c_int), ctypes.POINTER(ctypes.c_int)]
+        _lib = lib
+    return _lib
+
+
+class OracleError(RuntimeError):
+    def __init__(self, code: int):
+        super().__init__(f"oracle check failed ({code}): {ERRORS.get(code, '?')}")
+        self.code = code
+
+
+@dataclass
+class OracleResult:
+    P: int
+    root: int
+    nbytes: int
+    variant: int
+    scatter_size: int
+    schedule: np.ndarray      # (N, 9) int64, columns = FIELDS, canonical order
+    bytes_sent: np.ndarray    # (2, P) uint64: [phase, absolute rank]
+    bytes_recv: np.ndarray
+    msgs_sent: np.ndarray
+    msgs_recv: np.ndarray
+    bufs: np.ndarray | None   # (P, nbytes) uint8 after the broadcast, or None (schedule only)
+    seconds: float            # wall time of the simulation call alone
+
+    def col(self, name: str) -> np.ndarray:
+        return self.schedule[:, FIELDS.index(name)]
+
+    def phase_rows(self, phase: int) -> np.ndarray:
+        return self.schedule[self.col("phase") == phase]
+
+
+def scatter_size(P: int, nbytes: int) -> int:
+    return int(_load().oracle_bcast_scatter_size(P, nbytes))
+
+
+def step_flag(P: int, rel_rank: int) -> tuple[int, int]:
+    """(step, flag) of the tuned ring for one relative rank; flag is SEND_ONLY, RECV_ONLY or -1."""
+    step, flag = ctypes.c_int(), ctypes.c_int()
+    rc = _load().oracle_bcast_step_flag(P, rel_rank, ctypes.byref(step), ctypes.byref(flag))
+    if rc:
+        raise OracleError(rc)
+    return step.value, flag.value
+
+
+def capacity(P: int) -> int:
+    """Upper bound on the number of messages: P-1 scatter messages and P(P-1) ring messages."""
+    return max(1, (P - 1) + P * (P - 1))
+
+
+def simulate(P: int, root: int, nbytes: int, variant: int, message: np.ndarray | None = None,
+             bufs: np.ndarray | None = None) -> OracleResult:
+    """Run the simulated broadcast.
+
+    ``message``: uint8 array of ``nbytes`` (the root's data) -> per-rank buffers are created here,
+    non-root ones filled with a rank-dependent poison.  ``bufs``: a caller-made (P, nbytes) uint8
+    array used in place (the caller has put the message into ``bufs[root]``).  Neither: schedule
+    and counters only, no data moved.
+    """
+    lib = _load()
+    if bufs is None and message is not None:
+        message = np.ascontiguousarray(message, dtype=np.uint8)
+        assert message.shape == (nbytes,)
+        bufs = np.empty((P, nbytes), dtype=np.uint8)
+        for k in range(P):
+            bufs[k, :] = (0xA5 ^ (k * 37 + 11)) & 0xFF
+        bufs[root, :] = message
+    ptrs = None
+    if bufs is not None:
+        assert bufs.dtype == np.uint8 and bufs.shape == (P, nbytes) and bufs.flags.c_contiguous
+        base = bufs.ctypes.data
+        ptrs = (ctypes.c_void_p * P)(*[base + k * nbytes for k in range(P)])
+    cap = capacity(P)
+    sched = np.zeros((cap, len(FIELDS)), dtype=np.int64)
+    nsched = ctypes.c_int64(0)
+    cnt = [np.zeros((2, P), dtype=np.uint64) for _ in range(4)]
+    u64p = ctypes.POINTER(ctypes.c_uint64)
+    t0 = time.perf_counter()
+    rc = lib.oracle_bcast_simulate(
+        P, root, nbytes, variant, ptrs,
+        sched.ctypes.data_as(ctypes.POINTER(ctypes.c_int64)), cap, ctypes.byref(nsched),
+        *[c.ctypes.data_as(u64p) for c in cnt])
+    dt = time.perf_counter() - t0
+    if rc:
+        raise OracleError(rc)
+    return OracleResult(P=P, root=root, nbytes=nbytes, variant=variant,
+                        scatter_size=scatter_size(P, nbytes),
+                        schedule=sched[: nsched.value].copy(),
+                        bytes_sent=cnt[0], bytes_recv=cnt[1], msgs_sent=cnt[2], msgs_recv=cnt[3],
+                        bufs=bufs, seconds=dt)
