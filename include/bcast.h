@@ -1,0 +1,179 @@
+/*
+ * bcast.h -- C ABI of the scatter-ring-allgather broadcast over P virtual ranks whose
+ * receive buffers all live in the memory of one GPU.
+ *
+ * The method is the large-message / medium-message-non-power-of-two broadcast of MPICH as
+ * described in "A Bandwidth-saving Optimization for MPI Broadcast Collective Operation"
+ * (Zhou, Marjanovic, Niethammer, Gracia): the root's message is cut into P chunks of
+ * scatter_size = ceil(nbytes / P) bytes and scattered down a binomial tree (Section III-A,
+ * Figs. 1-2); a (P-1)-step ring allgather then completes every rank's buffer, either the
+ * NATIVE "enclosed" ring in which every rank receives in every step (Section III-A, Fig. 3)
+ * or the TUNED "non-enclosed" ring in which a rank never receives a chunk it already holds
+ * from the scatter (Section IV, Figs. 4-5 and the listing).
+ *
+ * bcast_plan()  turns that control flow into data: an ordered list of messages
+ *               (src_rank, dst_rank, chunk, offset, len) grouped into steps, plus per-rank
+ *               byte and message counters.  Host only, integers only.
+ * bcast_exec()  performs the messages of a plan as device-to-device copies between the P rank
+ *               buffers, honouring the step order: a byte is copied out of a rank's buffer only
+ *               after the message that delivers it to that rank has been performed.
+ *
+ * General conventions
+ *   - Every function returns BCAST_OK (0) or a negative BCAST_ERR_* code; nothing throws
+ *     across this boundary.  bcast_strerror() gives a static string for a code.
+ *   - "host" / "device" is stated for every pointer.  Ranks are ABSOLUTE ranks 0..P-1 unless a
+ *     field says "relative" (relative rank r = (rank - root + P) mod P, Section IV listing).
+ *   - A plan is immutable once created.  It may be executed any number of times; executions of
+ *     the same plan must not overlap in time on the GPU (the plan caches small device-side
+ *     tables and a work counter that executions share).
+ *   - The library keeps no other global state.  There is no CPU fallback: without a CUDA device
+ *     the bcast_exec* calls fail with BCAST_ERR_CUDA.
+ */
+#ifndef BCAST_B200_H
+#define BCAST_B200_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define BCAST_MAX_RANKS 1024 /* largest accepted P */
+
+enum { BCAST_NATIVE = 0, BCAST_TUNED = 1 };               /* variant: which ring allgather     */
+enum { BCAST_PHASE_SCATTER = 0, BCAST_PHASE_RING = 1 };   /* phase of a message                */
+
+enum {
+    BCAST_OK = 0,
+    BCAST_ERR_INVAL = -1,  /* bad argument (range, null, misaligned or overlapping buffers) */
+    BCAST_ERR_NOMEM = -2,  /* host or device allocation failed                              */
+    BCAST_ERR_CUDA = -3    /* a CUDA runtime call failed; see bcast_last_cuda_error()       */
+};
+
+/* How bcast_exec_mode() runs a plan.  All modes perform exactly the plan's messages. */
+enum {
+    /* One launch for the whole plan.  The message is cut into tiles on a fixed grid of byte
+       offsets; a thread block takes a tile and carries it through every message of the plan
+       that covers it, in plan order (scatter hops first, then ring hops), re-reading it from
+       the source rank's buffer at every hop.  Messages that cover different byte ranges are
+       independent, so no cross-block waiting is needed.  Default of bcast_exec(). */
+    BCAST_EXEC_WALK = 0,
+    /* One launch per plan step (ceil(log2 P) + P - 1 launches) on the caller's stream; inside a
+       launch the messages of that step are cut into tiles and copied in parallel. */
+    BCAST_EXEC_STEPS = 1,
+    /* The same per-step launches, captured once into a CUDA graph and replayed. */
+    BCAST_EXEC_GRAPH = 2
+};
+
+/* One message of the schedule.  Plain data, 48 bytes, host memory. */
+typedef struct {
+    int32_t phase;     /* BCAST_PHASE_SCATTER or BCAST_PHASE_RING                                   */
+    int32_t step;      /* scatter: tree level 0..L-1 (L = ceil(log2 P)); ring: i-1 for ring step i   */
+    int32_t src_rank;  /* absolute rank whose buffer is read                                        */
+    int32_t dst_rank;  /* absolute rank whose buffer is written                                     */
+    int32_t chunk;     /* RELATIVE index of the (first) chunk carried; chunk c = bytes
+                          [min(c*S, nbytes), min((c+1)*S, nbytes)) of the message                    */
+    int32_t nchunks;   /* ring: 1; scatter: the destination's own chunk plus its descendants'        */
+    uint64_t offset;   /* first byte, the same in the source and the destination buffer             */
+    uint64_t len;      /* bytes; 0 for chunks past the end of a short message (still a message)      */
+    int64_t dep;       /* index (into the plan's message array) of the message that last wrote this
+                          range into src_rank's buffer, -1 if it is the root's original data         */
+} bcast_xfer_t;
+
+typedef struct bcast_plan bcast_plan_t; /* opaque; created and freed by the library */
+
+/*
+ * bcast_plan -- build the schedule of one broadcast.
+ *   Scatter: Section III-A, Figs. 1-2 (binomial tree; L = ceil(log2 P) levels; in level t with
+ *   mask m = 2^(L-1-t) every relative rank r that is a multiple of 2m and has r+m < P sends the
+ *   chunks [r+m, min(r+2m, P)) to relative rank r+m).  Ring: Section III-A Fig. 3 (native) or
+ *   Section IV Figs. 4-5 and listing (tuned): in ring step i = 1..P-1 relative rank r receives
+ *   chunk (r-i) mod P from its left neighbour; in the tuned ring only while it still lacks it.
+ *   P        number of ranks, 1..BCAST_MAX_RANKS.  P = 1 gives an empty plan.
+ *   root     absolute rank that owns the message, 0..P-1
+ *   nbytes   message size; 0 is valid (all messages have len 0)
+ *   variant  BCAST_NATIVE or BCAST_TUNED
+ *   out      host pointer that receives the plan; the caller releases it with bcast_plan_free()
+ * Messages are ordered by (phase, step, dst_rank); a rank receives at most one message per step.
+ * Errors: BCAST_ERR_INVAL (arguments out of range, out == NULL), BCAST_ERR_NOMEM.
+ */
+int bcast_plan(int P, int root, uint64_t nbytes, int variant, bcast_plan_t **out);
+
+/* Release a plan and the device tables it cached (the device it was executed on must still be
+   usable).  NULL is ignored. */
+void bcast_plan_free(bcast_plan_t *plan);
+
+/* Read-only views of a plan.  All returned pointers are HOST pointers owned by the plan and
+   valid until bcast_plan_free(); a NULL plan (or a bad phase) gives 0 / NULL. */
+int32_t bcast_plan_num_ranks(const bcast_plan_t *plan);          /* P                               */
+int32_t bcast_plan_root(const bcast_plan_t *plan);
+int32_t bcast_plan_variant(const bcast_plan_t *plan);
+uint64_t bcast_plan_nbytes(const bcast_plan_t *plan);
+uint64_t bcast_plan_scatter_size(const bcast_plan_t *plan);      /* S = ceil(nbytes / P) (Section IV listing) */
+int64_t bcast_plan_num_xfers(const bcast_plan_t *plan);          /* number of messages               */
+int32_t bcast_plan_num_steps(const bcast_plan_t *plan);          /* L + (P-1); 0 for P = 1           */
+const bcast_xfer_t *bcast_plan_xfers(const bcast_plan_t *plan);  /* [num_xfers], canonical order      */
+const int64_t *bcast_plan_step_begin(const bcast_plan_t *plan);  /* [num_steps+1]: messages of step s
+                                                                    are [step_begin[s], step_begin[s+1]) */
+/* Per-rank counters of one phase, indexed by absolute rank, [P] each.  Message counts include
+   zero-length messages (Section IV counts ring messages this way: 56 vs 44 for P = 8). */
+const uint64_t *bcast_plan_bytes_sent(const bcast_plan_t *plan, int phase);
+const uint64_t *bcast_plan_bytes_recv(const bcast_plan_t *plan, int phase);
+const uint64_t *bcast_plan_msgs_sent(const bcast_plan_t *plan, int phase);
+const uint64_t *bcast_plan_msgs_recv(const bcast_plan_t *plan, int phase);
+uint64_t bcast_plan_total_bytes(const bcast_plan_t *plan);       /* sum of len over all messages      */
+
+/*
+ * bcast_exec -- perform a plan's messages on the GPU (Sections III-A and IV: the data movement
+ * of the scatter and of the ring allgather; every message is the copy of `len` bytes at `offset`
+ * from src_rank's buffer to the same offset of dst_rank's buffer).
+ *   rank_bufs    HOST array of P DEVICE pointers, one buffer of at least nbytes bytes per absolute
+ *                rank, all on the current device, 16-byte aligned, pairwise disjoint.  The array is
+ *                read before the call returns; the buffers stay owned by the caller.
+ *   plan         from bcast_plan()
+ *   cuda_stream  a cudaStream_t (NULL = the default stream).  The call only enqueues work and
+ *                does not synchronise; errors of the kernels themselves surface at the caller's
+ *                next synchronisation.
+ * On entry rank_bufs[root][0..nbytes) holds the message; other contents are arbitrary.  When the
+ * enqueued work has completed, rank_bufs[k][0..nbytes) equals the message for every k and no byte
+ * outside those ranges has been written.
+ * The first execution of a plan allocates and fills the plan's device tables (cudaMalloc and
+ * blocking copies); later executions allocate nothing.
+ * Errors: BCAST_ERR_INVAL (NULL arguments, NULL/misaligned/overlapping buffers, a device other
+ * than the one the plan was first executed on), BCAST_ERR_NOMEM, BCAST_ERR_CUDA.
+ */
+int bcast_exec(void *const *rank_bufs, const bcast_plan_t *plan, void *cuda_stream);
+
+/* bcast_exec with an explicit execution mode (BCAST_EXEC_*); same contract.  BCAST_EXEC_GRAPH
+   captures and instantiates its graph on the first call and again whenever rank_bufs differs
+   from the previous call. */
+int bcast_exec_mode(void *const *rank_bufs, const bcast_plan_t *plan, void *cuda_stream, int mode);
+
+/*
+ * bcast_exec_host -- the same broadcast for a caller whose data lives in HOST memory.
+ *   host_message  HOST pointer to nbytes bytes; copied into rank_bufs[root] first
+ *   host_out      HOST array of P HOST pointers (or NULL); after the broadcast the buffer of
+ *                 every rank k with host_out[k] != NULL is copied to host_out[k] (nbytes each)
+ *   rank_bufs, plan, cuda_stream, mode   as for bcast_exec_mode(); the device buffers are the
+ *                 working storage of the P ranks
+ * Copies use cudaMemcpyAsync on cuda_stream (pinned host memory makes them asynchronous and
+ * fast); the call returns after cudaStreamSynchronize, so on return host_out is filled.
+ * Errors: as bcast_exec, plus BCAST_ERR_INVAL for a NULL host_message when nbytes > 0.
+ */
+int bcast_exec_host(void *const *rank_bufs, const bcast_plan_t *plan, void *cuda_stream, int mode,
+                    const void *host_message, void *const *host_out);
+
+/* Number of kernel launches one execution of the plan enqueues in the given mode (0 if nothing
+   has to move); a CUDA-graph replay counts the kernels inside the graph. */
+int64_t bcast_exec_num_launches(const bcast_plan_t *plan, int mode);
+
+/* Static description of an error code. */
+const char *bcast_strerror(int code);
+
+/* The cudaError_t (as int) of the most recent failed CUDA call on this thread, 0 if none. */
+int bcast_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BCAST_B200_H */

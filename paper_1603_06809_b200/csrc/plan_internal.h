@@ -1,0 +1,22 @@
+// Internal layout of a plan, shared by the planner (plan.cpp) and the executor (exec.cu).
+#pragma once
+#include <cstdint>
+#include <vector>
+
+#include "bcast.h"
+
+struct bcast_device_state;   // defined in exec.cu; owns the device tables cached by a plan
+
+struct bcast_plan {
+    int P = 0, root = 0, variant = 0;
+    int L = 0;                                  // scatter levels, ceil(log2 P)
+    uint64_t nbytes = 0, S = 0;                 // message bytes, scatter_size
+    std::vector<bcast_xfer_t> xfers;            // canonical order: (phase, step, dst_rank)
+    std::vector<int64_t> step_begin;            // CSR over xfers, L + (P-1) + 1 entries
+    std::vector<uint64_t> bytes_sent[2], bytes_recv[2], msgs_sent[2], msgs_recv[2];   // [phase][rank]
+    uint64_t total_bytes = 0;
+    mutable bcast_device_state *dev = nullptr;  // created by the first execution
+};
+
+// exec.cu: frees the cached device tables of a plan (no-op when there are none)
+void bcast_device_state_free(bcast_device_state *dev);

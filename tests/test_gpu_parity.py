@@ -1,0 +1,197 @@
+"""GPU parity: the CUDA executors, called through the C ABI, against the CPU oracle.
+
+Byte work, so the bar is bit-exact: every rank buffer equals the oracle's buffer of that rank
+element by element, guard zones around the buffers are untouched, and the plan that was executed
+equals the oracle's schedule and counters (tests/test_plan_parity.py checks the latter on CPU)."""
+import ctypes
+
+import numpy as np
+import pytest
+import torch
+
+from paper_1603_06809_b200 import bcast as B
+from paper_1603_06809_b200 import workloads as W
+from gpu_harness import RankBuffers, run_broadcast
+
+pytestmark = pytest.mark.gpu
+
+MODES = [B.BCAST_EXEC_WALK, B.BCAST_EXEC_STEPS, B.BCAST_EXEC_GRAPH]
+MODE_IDS = ["walk", "steps", "graph"]
+VARIANTS = [B.BCAST_NATIVE, B.BCAST_TUNED]
+VARIANT_IDS = ["native", "tuned"]
+
+
+def check_against_oracle(oracle, wl, variant, mode, shift=0, repeats=1):
+    msg = W.message_bytes(wl.seed, wl.nbytes)
+    plan, bufs = run_broadcast(wl.P, wl.root, wl.nbytes, variant, mode, msg, shift=shift, repeats=repeats)
+    ref = oracle.simulate(wl.P, wl.root, wl.nbytes, variant, message=msg)
+    got = bufs.to_host()
+    assert got.shape == ref.bufs.shape
+    assert np.array_equal(got, ref.bufs)
+    assert bufs.guards_intact()
+    x = B.bcast_plan_xfers(plan)
+    assert len(x) == len(ref.schedule)
+    assert np.array_equal(x["len"].astype(np.int64), ref.col("len"))
+    assert np.array_equal(x["src_rank"].astype(np.int64), ref.col("src"))
+    assert np.array_equal(x["dst_rank"].astype(np.int64), ref.col("dst"))
+    assert np.array_equal(x["offset"].astype(np.int64), ref.col("offset"))
+    for ph in (0, 1):
+        assert np.array_equal(B.bcast_plan_bytes_recv(plan, ph), ref.bytes_recv[ph])
+        assert np.array_equal(B.bcast_plan_bytes_sent(plan, ph), ref.bytes_sent[ph])
+
+
+# ---- configurations 1-3 in full, element by element, all executors
+@pytest.mark.parametrize("mode", MODES, ids=MODE_IDS)
+@pytest.mark.parametrize("variant", VARIANTS, ids=VARIANT_IDS)
+@pytest.mark.parametrize("wl", [W.CFG1, W.CFG2, W.CFG3], ids=lambda w: w.name)
+def test_configs_1_to_3(oracle, wl, variant, mode):
+    check_against_oracle(oracle, wl, variant, mode)
+
+
+# ---- configuration 2 with every root
+@pytest.mark.parametrize("variant", VARIANTS, ids=VARIANT_IDS)
+def test_cfg2_all_roots(oracle, variant):
+    for wl in W.cfg2_all_roots():
+        check_against_oracle(oracle, wl, variant, B.BCAST_EXEC_WALK)
+    check_against_oracle(oracle, W.cfg2_all_roots()[7], variant, B.BCAST_EXEC_STEPS)
+
+
+# ---- small, ragged and degenerate shapes: several tiles plus ragged tails, chunks shorter than a
+# word, empty chunks, nbytes < P, nbytes = 0, P = 1, P = 2
+SMALL = [(1, 0, 1000), (2, 1, 1), (2, 0, 4097), (3, 1, 2), (5, 3, 4), (7, 6, 12288), (9, 4, 524287),
+         (10, 0, 40), (16, 15, 65521), (17, 5, 1048576), (33, 32, 100003), (255, 254, 12288),
+         (256, 255, 12288), (13, 2, 13 * 16 * 256 * 4 + 5), (6, 2, 0), (64, 63, 63), (129, 77, 2560000)]
+
+
+@pytest.mark.parametrize("mode", MODES, ids=MODE_IDS)
+@pytest.mark.parametrize("variant", VARIANTS, ids=VARIANT_IDS)
+@pytest.mark.parametrize("P,root,n", SMALL)
+def test_small_and_ragged(oracle, P, root, n, variant, mode):
+    check_against_oracle(oracle, W.Workload(f"P{P}_{n}", P, root, n, 7000 + P), variant, mode)
+
+
+@pytest.mark.parametrize("mode", MODES, ids=MODE_IDS)
+def test_buffers_at_odd_16_byte_offsets(oracle, mode):
+    """Rank buffers only need 16-byte alignment, not more."""
+    for shift in (16, 48, 240):
+        check_against_oracle(oracle, W.Workload("shifted", 12, 5, 100001, 99), B.BCAST_TUNED, mode, shift=shift)
+
+
+@pytest.mark.parametrize("mode", MODES, ids=MODE_IDS)
+def test_repeated_execution_and_new_buffers(oracle, mode):
+    """A plan can be executed again (work counters return to zero) and with other buffers."""
+    wl = W.Workload("again", 24, 23, 4 * W.MiB + 3, 123)
+    check_against_oracle(oracle, wl, B.BCAST_TUNED, mode, repeats=3)
+    msg = W.message_bytes(wl.seed, wl.nbytes)
+    plan = B.bcast_plan(wl.P, wl.root, wl.nbytes, B.BCAST_NATIVE)
+    for rep in range(2):
+        bufs = RankBuffers(wl.P, wl.root, wl.nbytes, msg, shift=16 * rep)
+        B.bcast_exec_mode(bufs.pointers(), plan, torch.cuda.current_stream(), mode)
+        torch.cuda.synchronize()
+        assert bufs.all_equal_message() and bufs.guards_intact()
+
+
+def test_runs_on_a_side_stream(oracle):
+    wl = W.Workload("side", 12, 3, 3 * W.MiB + 1, 5)
+    msg = W.message_bytes(wl.seed, wl.nbytes)
+    bufs = RankBuffers(wl.P, wl.root, wl.nbytes, msg)
+    plan = B.bcast_plan(wl.P, wl.root, wl.nbytes, B.BCAST_TUNED)
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    for mode in MODES:
+        bufs.reset()
+        torch.cuda.synchronize()
+        B.bcast_exec_mode(bufs.pointers(), plan, side, mode)
+        side.synchronize()
+        assert bufs.all_equal_message() and bufs.guards_intact()
+
+
+# ---- configuration 4 at full size, in the launch configuration the benchmark times (WALK): every
+# rank buffer compared with the root's message on the device, sampled ranks against the oracle's
+# buffers on the host, schedule and counters against the oracle
+@pytest.mark.parametrize("variant", VARIANTS, ids=VARIANT_IDS)
+def test_cfg4_full_size(oracle, variant):
+    wl = W.CFG4
+    msg = W.message_bytes(wl.seed, wl.nbytes)
+    plan, bufs = run_broadcast(wl.P, wl.root, wl.nbytes, variant, B.BCAST_EXEC_WALK, msg)
+    assert bufs.all_equal_message() and bufs.guards_intact()
+    ref = oracle.simulate(wl.P, wl.root, wl.nbytes, variant, message=msg)
+    for k in (0, 1, 37, 62, 63, 64, 99):
+        assert np.array_equal(bufs.view[k].cpu().numpy(), ref.bufs[k])
+    x = B.bcast_plan_xfers(plan)
+    assert np.array_equal(x["len"].astype(np.int64), ref.col("len"))
+    assert B.bcast_plan_total_bytes(plan) == int(ref.col("len").sum())
+
+
+def test_cfg4_steps_executor():
+    wl = W.CFG4
+    msg = W.message_bytes(wl.seed, wl.nbytes)
+    _, bufs = run_broadcast(wl.P, wl.root, wl.nbytes, B.BCAST_TUNED, B.BCAST_EXEC_GRAPH, msg)
+    assert bufs.all_equal_message() and bufs.guards_intact()
+
+
+# ---- configuration 5: the sweep.  Points the oracle finishes in seconds are compared element by
+# element on the host; the large ones (up to 34 GB of rank buffers) rank by rank against the
+# message on the device, which is what the oracle's buffers equal (MPI broadcast semantics).
+@pytest.mark.parametrize("variant", VARIANTS, ids=VARIANT_IDS)
+def test_sweep(oracle, variant):
+    for wl in W.sweep():
+        if wl.total_bytes <= 600 * W.MiB:
+            check_against_oracle(oracle, wl, variant, B.BCAST_EXEC_WALK)
+        else:
+            msg = W.message_bytes(wl.seed, wl.nbytes)
+            plan, bufs = run_broadcast(wl.P, wl.root, wl.nbytes, variant, B.BCAST_EXEC_WALK, msg)
+            assert bufs.all_equal_message() and bufs.guards_intact(), wl.name
+            ref = oracle.simulate(wl.P, wl.root, wl.nbytes, variant)          # schedule and counters only
+            assert B.bcast_plan_total_bytes(plan) == int(ref.col("len").sum())
+            del bufs
+            torch.cuda.empty_cache()
+
+
+def test_sweep_steps_executor_medium_points(oracle):
+    for wl in W.sweep():
+        if wl.total_bytes <= 128 * W.MiB:
+            check_against_oracle(oracle, wl, B.BCAST_TUNED, B.BCAST_EXEC_STEPS)
+
+
+# ---- host-memory entry point
+@pytest.mark.parametrize("variant", VARIANTS, ids=VARIANT_IDS)
+def test_exec_host(oracle, variant):
+    wl = W.Workload("host", 12, 5, 1 * W.MiB + 77, 31)
+    msg = W.message_bytes(wl.seed, wl.nbytes)
+    bufs = RankBuffers(wl.P, wl.root, wl.nbytes, np.zeros(wl.nbytes, np.uint8))   # root NOT pre-filled
+    plan = B.bcast_plan(wl.P, wl.root, wl.nbytes, variant)
+    host_msg = torch.from_numpy(msg.copy()).pin_memory()
+    outs = torch.zeros((wl.P, wl.nbytes), dtype=torch.uint8).pin_memory()
+    out_list = [outs[k] for k in range(wl.P)]
+    out_list[3] = None
+    B.bcast_exec_host(bufs.pointers(), plan, torch.cuda.current_stream(), B.BCAST_EXEC_WALK, host_msg, out_list)
+    ref = oracle.simulate(wl.P, wl.root, wl.nbytes, variant, message=msg)
+    got = outs.numpy()
+    for k in range(wl.P):
+        if k == 3:
+            assert not got[k].any()
+        else:
+            assert np.array_equal(got[k], ref.bufs[k])
+    assert bufs.guards_intact()
+
+
+# ---- argument errors are refused before anything is launched
+def test_exec_rejects_bad_buffers():
+    wl = W.Workload("bad", 4, 0, 4096, 1)
+    msg = W.message_bytes(wl.seed, wl.nbytes)
+    bufs = RankBuffers(wl.P, wl.root, wl.nbytes, msg)
+    plan = B.bcast_plan(wl.P, wl.root, wl.nbytes, B.BCAST_TUNED)
+    good = bufs.pointers()
+    for bad in ([good[0], 0, good[2], good[3]],                  # NULL
+                [good[0], good[1] + 8, good[2], good[3]],        # misaligned
+                [good[0], good[1], good[1], good[3]],            # duplicate
+                [good[0], good[0] + 1024, good[2], good[3]]):    # overlapping
+        with pytest.raises(B.BcastError) as e:
+            B.bcast_exec(bad, plan)
+        assert e.value.code == B.BCAST_ERR_INVAL
+    torch.cuda.synchronize()
+    assert not bufs.all_equal_message()          # nothing ran
+    B.bcast_exec(good, plan)
+    torch.cuda.synchronize()
+    assert bufs.all_equal_message() and bufs.guards_intact()

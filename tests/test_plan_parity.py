@@ -1,0 +1,133 @@
+"""Host-side checks without a GPU: the library loads and exports every symbol of include/bcast.h,
+and the planner's schedule, dependency indices and per-rank counters equal the oracle's
+bit for bit (the planner uses the closed form of the binomial tree, the oracle runs the
+per-process loops of the paper's listing: two derivations of the same schedule)."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+from helpers import ROOT
+from paper_1603_06809_b200 import bcast as B
+from paper_1603_06809_b200 import workloads as W
+
+FIELDS = ("phase", "step", "src_rank", "dst_rank", "chunk", "nchunks", "offset", "len", "dep")
+
+
+def plan_matrix(plan):
+    x = B.bcast_plan_xfers(plan)
+    return np.stack([x[f].astype(np.int64) for f in FIELDS], axis=1) if len(x) else np.zeros((0, 9), np.int64)
+
+
+def assert_plan_equals_oracle(oracle, P, root, n, variant):
+    plan = B.bcast_plan(P, root, n, variant)
+    ref = oracle.simulate(P, root, n, variant)
+    mine = plan_matrix(plan)
+    assert mine.shape == ref.schedule.shape
+    assert (mine == ref.schedule).all()
+    assert B.bcast_plan_scatter_size(plan) == ref.scatter_size
+    assert B.bcast_plan_total_bytes(plan) == int(ref.col("len").sum())
+    for ph in (B.BCAST_PHASE_SCATTER, B.BCAST_PHASE_RING):
+        assert (B.bcast_plan_bytes_sent(plan, ph) == ref.bytes_sent[ph]).all()
+        assert (B.bcast_plan_bytes_recv(plan, ph) == ref.bytes_recv[ph]).all()
+        assert (B.bcast_plan_msgs_sent(plan, ph) == ref.msgs_sent[ph]).all()
+        assert (B.bcast_plan_msgs_recv(plan, ph) == ref.msgs_recv[ph]).all()
+    # CSR over steps: L + P - 1 steps, each holding the messages with that (phase, step)
+    sb = B.bcast_plan_step_begin(plan)
+    L = (P - 1).bit_length()
+    nsteps = L + P - 1 if P > 1 else 0
+    assert B.bcast_plan_num_steps(plan) == nsteps and len(sb) == nsteps + 1
+    assert sb[0] == 0 and sb[-1] == len(mine) and (np.diff(sb) >= 0).all()
+    for s in range(nsteps):
+        rows = mine[sb[s]:sb[s + 1]]
+        want = (0, s) if s < L else (1, s - L)
+        assert ((rows[:, 0] == want[0]) & (rows[:, 1] == want[1])).all()
+    B.bcast_plan_free(plan)
+
+
+def test_library_exports_every_declared_symbol():
+    header = open(os.path.join(ROOT, "include", "bcast.h")).read()
+    declared = set(re.findall(r"\b(bcast_[a-z_]+)\s*\(", header))
+    assert declared == set(B.SYMBOLS)
+    lib = ctypes.CDLL(os.path.join(ROOT, "paper_1603_06809_b200", "libbcast_b200.so"))
+    for name in declared:
+        assert hasattr(lib, name), name
+
+
+def test_xfer_layout_matches_header():
+    assert B.XFER_DTYPE.itemsize == 48
+    assert [B.XFER_DTYPE.fields[f][1] for f in FIELDS] == [0, 4, 8, 12, 16, 20, 24, 32, 40]
+
+
+@pytest.mark.parametrize("variant", [B.BCAST_NATIVE, B.BCAST_TUNED])
+def test_plan_equals_oracle_small_grid(oracle, variant):
+    for P in list(range(1, 34)) + [63, 64, 65]:
+        for root in sorted({0, P // 3, P - 1}):
+            for n in (0, 1, P - 1, P, P + 1, 97, 12288, 1000003):
+                assert_plan_equals_oracle(oracle, P, root, n, variant)
+
+
+@pytest.mark.parametrize("variant", [B.BCAST_NATIVE, B.BCAST_TUNED])
+@pytest.mark.parametrize("wl", [W.CFG1, W.CFG2, W.CFG3, W.CFG4], ids=lambda w: w.name)
+def test_plan_equals_oracle_configs(oracle, wl, variant):
+    assert_plan_equals_oracle(oracle, wl.P, wl.root, wl.nbytes, variant)
+
+
+@pytest.mark.parametrize("variant", [B.BCAST_NATIVE, B.BCAST_TUNED])
+def test_plan_equals_oracle_all_roots_cfg2(oracle, variant):
+    for wl in W.cfg2_all_roots():
+        assert_plan_equals_oracle(oracle, wl.P, wl.root, wl.nbytes, variant)
+
+
+@pytest.mark.parametrize("variant", [B.BCAST_NATIVE, B.BCAST_TUNED])
+def test_plan_equals_oracle_sweep(oracle, variant):
+    sweep = W.sweep()
+    assert len(sweep) == 45
+    for wl in sweep:
+        assert_plan_equals_oracle(oracle, wl.P, wl.root, wl.nbytes, variant)
+
+
+def test_plan_largest_rank_count(oracle):
+    assert_plan_equals_oracle(oracle, B.BCAST_MAX_RANKS, 1000, 5_000_011, B.BCAST_TUNED)
+
+
+def test_plan_argument_errors():
+    for args in [(0, 0, 10, 1), (-1, 0, 10, 1), (B.BCAST_MAX_RANKS + 1, 0, 10, 1), (4, 4, 10, 1), (4, -1, 10, 1),
+                 (4, 0, 10, 2), (4, 0, 10, -1), (4, 0, 2**64 - 1, 1)]:
+        with pytest.raises(B.BcastError) as e:
+            B.bcast_plan(*args)
+        assert e.value.code == B.BCAST_ERR_INVAL
+    # out == NULL
+    assert B._lib.bcast_plan(4, 0, 10, 1, None) == B.BCAST_ERR_INVAL
+    # NULL plan: accessors answer 0 / NULL, free is a no-op
+    assert B._lib.bcast_plan_num_xfers(None) == 0 and not B._lib.bcast_plan_xfers(None)
+    assert not B._lib.bcast_plan_bytes_sent(None, 0)
+    B._lib.bcast_plan_free(None)
+    plan = B.bcast_plan(4, 0, 10, 1)
+    assert not B._lib.bcast_plan_bytes_sent(plan.handle, 2)
+    assert B.bcast_strerror(B.BCAST_ERR_INVAL) == "invalid argument" and B.bcast_strerror(0) == "success"
+
+
+def test_exec_argument_errors_need_no_gpu():
+    plan = B.bcast_plan(4, 0, 64, 1)
+    assert B._lib.bcast_exec(None, plan.handle, None) == B.BCAST_ERR_INVAL
+    assert B._lib.bcast_exec((ctypes.c_void_p * 4)(16, 32, 48, 64), None, None) == B.BCAST_ERR_INVAL
+    assert B._lib.bcast_exec_mode((ctypes.c_void_p * 4)(16, 32, 48, 64), plan.handle, None, 7) == B.BCAST_ERR_INVAL
+    assert B.bcast_exec_num_launches(plan, B.BCAST_EXEC_WALK) == 1
+    assert B.bcast_exec_num_launches(plan, B.BCAST_EXEC_STEPS) == 2 + 3
+    assert B.bcast_exec_num_launches(B.bcast_plan(1, 0, 64, 1), B.BCAST_EXEC_WALK) == 0
+    assert B.bcast_exec_num_launches(B.bcast_plan(4, 0, 0, 1), B.BCAST_EXEC_STEPS) == 0
+    # P = 255, 12 KiB: the last four chunks are empty, but every step still moves something
+    assert B.bcast_exec_num_launches(B.bcast_plan(255, 254, 12288, 0), B.BCAST_EXEC_STEPS) == 8 + 254
+
+
+def test_exec_without_gpu_fails_loudly():
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("a GPU is present")
+    plan = B.bcast_plan(4, 0, 64, 1)
+    with pytest.raises(B.BcastError) as e:
+        B.bcast_exec([4096, 8192, 12288, 16384], plan)
+    assert e.value.code == B.BCAST_ERR_CUDA
