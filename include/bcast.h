@@ -47,7 +47,8 @@ enum {
     BCAST_OK = 0,
     BCAST_ERR_INVAL = -1,  /* bad argument (range, null, misaligned or overlapping buffers) */
     BCAST_ERR_NOMEM = -2,  /* host or device allocation failed                              */
-    BCAST_ERR_CUDA = -3    /* a CUDA runtime call failed; see bcast_last_cuda_error()       */
+    BCAST_ERR_CUDA = -3,   /* a CUDA runtime call failed; see bcast_last_cuda_error()       */
+    BCAST_ERR_CAPACITY = -4 /* bcast_exec_static only: the plan's tables exceed the built-in scratch */
 };
 
 /* How bcast_exec_mode() runs a plan.  All modes perform exactly the plan's messages. */
@@ -162,6 +163,38 @@ int bcast_exec_mode(void *const *rank_bufs, const bcast_plan_t *plan, void *cuda
  */
 int bcast_exec_host(void *const *rank_bufs, const bcast_plan_t *plan, void *cuda_stream, int mode,
                     const void *host_message, void *const *host_out);
+
+/*
+ * bcast_exec_static -- bcast_exec for callers that must not allocate device memory.
+ * (The paper has no counterpart to this entry point; it exists for the sake of such callers.)
+ *
+ * Who needs it: programs that hand all device memory to their own pool at start-up and may not
+ * call cudaMalloc afterwards (a raw allocation can fail or fragment the pool's address space),
+ * services that run under a fixed memory budget, and latency-critical code for which the implicit
+ * device-wide synchronisation of cudaMalloc / cudaFree is not acceptable.  bcast_exec() allocates
+ * the plan's device tables on a plan's first execution; this call never allocates: it runs the
+ * same one-launch WALK kernel, with the tables it needs (tile list, per-chunk hop lists, work
+ * counter) placed in a fixed array of BCAST_STATIC_SCRATCH_BYTES bytes that is part of the
+ * library's device image.  Every GPU on which the library is loaded holds that array until the
+ * process exits.
+ *   rank_bufs, plan, cuda_stream   as for bcast_exec(); inputs and outputs are still the caller's.
+ * Behaviour to know about:
+ *   - Plans whose tables do not fit (roughly: 24 B per 4..32 KiB tile of the message plus 4 B per
+ *     (chunk, message) pair, about 4*P*P bytes) are refused with BCAST_ERR_CAPACITY before
+ *     anything is copied or launched.  All configurations up to P = 256 ranks with messages up to
+ *     512 MiB fit; P = 1024 does not.
+ *   - The first call on a device looks up the array's device address (cudaGetSymbolAddress) and
+ *     remembers it; make that first call outside any stream capture.
+ *   - Every call re-writes the array (stream-ordered on cuda_stream) from host memory, including
+ *     the work counter that has to start at zero, so the array's previous contents never matter.
+ *     Because all calls share the one array, two calls whose GPU work overlaps in time (different
+ *     streams, or different host threads) race on it: serialise them.
+ *   - No cudaMalloc, cudaFree or other allocating CUDA call is made; ordinary host heap memory is
+ *     used briefly to assemble the tables.
+ * Errors: BCAST_ERR_INVAL as for bcast_exec, BCAST_ERR_CAPACITY, BCAST_ERR_CUDA.
+ */
+#define BCAST_STATIC_SCRATCH_BYTES (2u << 20)
+int bcast_exec_static(void *const *rank_bufs, const bcast_plan_t *plan, void *cuda_stream);
 
 /* Number of kernel launches one execution of the plan enqueues in the given mode (0 if nothing
    has to move); a CUDA-graph replay counts the kernels inside the graph. */

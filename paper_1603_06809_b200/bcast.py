@@ -21,7 +21,8 @@ _lib = ctypes.CDLL(_LIB_PATH)
 BCAST_MAX_RANKS = 1024
 BCAST_NATIVE, BCAST_TUNED = 0, 1
 BCAST_PHASE_SCATTER, BCAST_PHASE_RING = 0, 1
-BCAST_OK, BCAST_ERR_INVAL, BCAST_ERR_NOMEM, BCAST_ERR_CUDA = 0, -1, -2, -3
+BCAST_OK, BCAST_ERR_INVAL, BCAST_ERR_NOMEM, BCAST_ERR_CUDA, BCAST_ERR_CAPACITY = 0, -1, -2, -3, -4
+BCAST_STATIC_SCRATCH_BYTES = 2 << 20
 BCAST_EXEC_WALK, BCAST_EXEC_STEPS, BCAST_EXEC_GRAPH = 0, 1, 2
 
 #: numpy view of ``bcast_xfer_t`` (48 bytes)
@@ -36,7 +37,7 @@ SYMBOLS = (
     "bcast_plan_nbytes", "bcast_plan_scatter_size", "bcast_plan_num_xfers", "bcast_plan_num_steps",
     "bcast_plan_xfers", "bcast_plan_step_begin", "bcast_plan_bytes_sent", "bcast_plan_bytes_recv",
     "bcast_plan_msgs_sent", "bcast_plan_msgs_recv", "bcast_plan_total_bytes", "bcast_exec",
-    "bcast_exec_mode", "bcast_exec_host", "bcast_exec_num_launches", "bcast_strerror",
+    "bcast_exec_mode", "bcast_exec_host", "bcast_exec_static", "bcast_exec_num_launches", "bcast_strerror",
     "bcast_last_cuda_error",
 )
 
@@ -55,6 +56,7 @@ _sig = {
     "bcast_exec": (_i, [_vpp, _vp, _vp]),
     "bcast_exec_mode": (_i, [_vpp, _vp, _vp, _i]),
     "bcast_exec_host": (_i, [_vpp, _vp, _vp, _i, _vp, _vpp]),
+    "bcast_exec_static": (_i, [_vpp, _vp, _vp]),
     "bcast_exec_num_launches": (_i64, [_vp, _i]),
     "bcast_strerror": (ctypes.c_char_p, [_i]),
     "bcast_last_cuda_error": (_i, []),
@@ -205,6 +207,19 @@ def bcast_exec_host(rank_bufs, plan: Plan, stream, mode: int, host_message, host
     outs = None if host_out is None else (ctypes.c_void_p * P)(*[host_ptr(x) for x in host_out])
     _check(_lib.bcast_exec_host(_ptr_array(rank_bufs, "rank_bufs"), plan.handle, _stream_ptr(stream), mode,
                                 ctypes.c_void_p(host_ptr(host_message)), outs), "bcast_exec_host")
+
+
+def bcast_exec_static(rank_bufs, plan: Plan, stream=None) -> None:
+    """The broadcast for callers that must not allocate device memory (memory handed to a pool,
+    fixed budgets, no tolerance for cudaMalloc's device-wide synchronisation): same arguments as
+    :func:`bcast_exec`; the kernel's tables go into a fixed array inside the library instead of
+    memory from cudaMalloc.  Raises ``BcastError`` with ``BCAST_ERR_CAPACITY`` when the plan's
+    tables exceed ``BCAST_STATIC_SCRATCH_BYTES``.  Calls share that array: do not let two of them
+    overlap on the GPU."""
+    if len(rank_bufs) != bcast_plan_num_ranks(plan):
+        raise BcastError(BCAST_ERR_INVAL, "bcast_exec_static (len(rank_bufs) != P)")
+    _check(_lib.bcast_exec_static(_ptr_array(rank_bufs, "rank_bufs"), plan.handle, _stream_ptr(stream)),
+           "bcast_exec_static")
 
 
 def bcast_exec_num_launches(plan: Plan, mode: int = BCAST_EXEC_WALK) -> int:

@@ -23,6 +23,7 @@
 #include <algorithm>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -311,8 +312,15 @@ int build_step_tables(const bcast_plan_t &p, bcast_device_state &ds)
     return upload(&ds.d_xfers, hx);
 }
 
-// Tables of the WALK executor: per chunk the list of (src, dst) hops in plan order, and the tiles.
-int build_walk_tables(const bcast_plan_t &p, bcast_device_state &ds)
+// Host form of the WALK executor's tables: per chunk the list of (src, dst) hops in plan order,
+// and the tiles (fixed grid of `256 * u * 16`-byte offsets, split at chunk boundaries).
+struct WalkTables {
+    std::vector<WalkItem> items;
+    std::vector<uint32_t> hops;
+    std::vector<int> hop_begin;   // [P + 1], by relative chunk index
+};
+
+int make_walk_tables(const bcast_plan_t &p, int u, WalkTables &t)
 {
     const int P = p.P;
     auto chunk_begin = [&](int c) { return std::min<uint64_t>((uint64_t)c * p.S, p.nbytes); };
@@ -323,51 +331,63 @@ int build_walk_tables(const bcast_plan_t &p, bcast_device_state &ds)
         for (int c = x.chunk; c < x.chunk + x.nchunks; c++)
             if (chunk_begin(c + 1) > chunk_begin(c)) per_chunk[c].push_back(e);
     }
-    std::vector<int> hop_begin(P + 1, 0);
-    std::vector<uint32_t> hops;
+    t.hop_begin.assign(P + 1, 0);
+    t.hops.clear();
     for (int c = 0; c < P; c++) {
         if ((int)per_chunk[c].size() > kMaxHops) return BCAST_ERR_INVAL;
-        hop_begin[c] = (int)hops.size();
-        hops.insert(hops.end(), per_chunk[c].begin(), per_chunk[c].end());
+        t.hop_begin[c] = (int)t.hops.size();
+        t.hops.insert(t.hops.end(), per_chunk[c].begin(), per_chunk[c].end());
     }
-    hop_begin[P] = (int)hops.size();
+    t.hop_begin[P] = (int)t.hops.size();
 
-    // words per thread: large tiles when the message is big enough to fill the GPU with them
-    int bps = 1;
-    int u = env_int("BCAST_WALK_WORDS", 0);
-    if (u != 1 && u != 2 && u != 4 && u != 8) {
-        u = 1;
-        for (int cand : {4, 2}) {
-            const uint64_t tile = (uint64_t)kThreads * cand * 16;
-            if (p.nbytes / tile >= (uint64_t)ds.sm_count * 8) { u = cand; break; }
-        }
-    }
-    ds.walk_u = u;
     const uint64_t tile = (uint64_t)kThreads * u * 16;
-    std::vector<WalkItem> items;
+    t.items.clear();
     for (int c = 0; c < P; c++) {
         const uint64_t b = chunk_begin(c), e = chunk_begin(c + 1);
         if (e <= b || per_chunk[c].empty()) continue;
-        for (uint64_t t = b / tile; t * tile < e; t++)
-            items.push_back(WalkItem{std::max(b, t * tile), std::min(e, (t + 1) * tile), c, 0});
+        for (uint64_t g = b / tile; g * tile < e; g++)
+            t.items.push_back(WalkItem{std::max(b, g * tile), std::min(e, (g + 1) * tile), c, 0});
     }
-    ds.n_items = (int)items.size();
+    return BCAST_OK;
+}
 
-    int rc;
-    if (P <= 128) {
-        rc = u == 8 ? walk_occupancy<8, 128>(&bps) : u == 4 ? walk_occupancy<4, 128>(&bps)
-           : u == 2 ? walk_occupancy<2, 128>(&bps) : walk_occupancy<1, 128>(&bps);
-    } else {
-        rc = u == 8 ? walk_occupancy<8, BCAST_MAX_RANKS>(&bps) : u == 4 ? walk_occupancy<4, BCAST_MAX_RANKS>(&bps)
-           : u == 2 ? walk_occupancy<2, BCAST_MAX_RANKS>(&bps) : walk_occupancy<1, BCAST_MAX_RANKS>(&bps);
+// words per thread: large tiles when the message is big enough to fill the GPU with them
+int choose_walk_words(uint64_t nbytes, int sm_count)
+{
+    const int forced = env_int("BCAST_WALK_WORDS", 0);
+    if (forced == 1 || forced == 2 || forced == 4 || forced == 8) return forced;
+    for (int cand : {4, 2}) {
+        const uint64_t tile = (uint64_t)kThreads * cand * 16;
+        if (nbytes / tile >= (uint64_t)sm_count * 8) return cand;
     }
+    return 1;
+}
+
+int walk_blocks_per_sm(int u, int P, int *bps)
+{
+    if (P <= 128)
+        return u == 8 ? walk_occupancy<8, 128>(bps) : u == 4 ? walk_occupancy<4, 128>(bps)
+             : u == 2 ? walk_occupancy<2, 128>(bps) : walk_occupancy<1, 128>(bps);
+    return u == 8 ? walk_occupancy<8, BCAST_MAX_RANKS>(bps) : u == 4 ? walk_occupancy<4, BCAST_MAX_RANKS>(bps)
+         : u == 2 ? walk_occupancy<2, BCAST_MAX_RANKS>(bps) : walk_occupancy<1, BCAST_MAX_RANKS>(bps);
+}
+
+// Device tables of the WALK executor, cached in the plan's device state.
+int build_walk_tables(const bcast_plan_t &p, bcast_device_state &ds)
+{
+    ds.walk_u = choose_walk_words(p.nbytes, ds.sm_count);
+    WalkTables t;
+    int rc = make_walk_tables(p, ds.walk_u, t);
     if (rc) return rc;
+    ds.n_items = (int)t.items.size();
+    int bps = 1;
+    if ((rc = walk_blocks_per_sm(ds.walk_u, p.P, &bps))) return rc;
     const int cap = env_int("BCAST_WALK_BLOCKS_PER_SM", bps);
     ds.walk_grid = std::max(1, std::min(ds.n_items, ds.sm_count * std::max(1, std::min(cap, bps))));
 
-    if ((rc = upload(&ds.d_items, items))) return rc;
-    if ((rc = upload(&ds.d_hops, hops))) return rc;
-    if ((rc = upload(&ds.d_hop_begin, hop_begin))) return rc;
+    if ((rc = upload(&ds.d_items, t.items))) return rc;
+    if ((rc = upload(&ds.d_hops, t.hops))) return rc;
+    if ((rc = upload(&ds.d_hop_begin, t.hop_begin))) return rc;
     CUDA_TRY(cudaMalloc((void **)&ds.d_ctl, sizeof(WalkCtl)));
     CUDA_TRY(cudaMemset(ds.d_ctl, 0, sizeof(WalkCtl)));
     return BCAST_OK;
@@ -401,11 +421,8 @@ int get_state(const bcast_plan_t &p, bcast_device_state **out)
 }
 
 // NULL, misaligned or overlapping rank buffers are refused before anything is launched.
-int check_bufs(void *const *rank_bufs, const bcast_plan_t &p, bcast_device_state &ds)
+int validate_bufs(void *const *rank_bufs, size_t P, uint64_t nbytes)
 {
-    const size_t P = (size_t)p.P;
-    if (ds.checked_bufs.size() == P && std::memcmp(ds.checked_bufs.data(), rank_bufs, P * sizeof(void *)) == 0)
-        return BCAST_OK;
     std::vector<uintptr_t> a(P);
     for (size_t k = 0; k < P; k++) {
         a[k] = (uintptr_t)rank_bufs[k];
@@ -413,7 +430,18 @@ int check_bufs(void *const *rank_bufs, const bcast_plan_t &p, bcast_device_state
     }
     std::sort(a.begin(), a.end());
     for (size_t k = 1; k < P; k++)
-        if (a[k] - a[k - 1] < std::max<uint64_t>(p.nbytes, 1)) return BCAST_ERR_INVAL;
+        if (a[k] - a[k - 1] < std::max<uint64_t>(nbytes, 1)) return BCAST_ERR_INVAL;
+    return BCAST_OK;
+}
+
+// The same check, skipped when the pointers are the ones that passed it last time.
+int check_bufs(void *const *rank_bufs, const bcast_plan_t &p, bcast_device_state &ds)
+{
+    const size_t P = (size_t)p.P;
+    if (ds.checked_bufs.size() == P && std::memcmp(ds.checked_bufs.data(), rank_bufs, P * sizeof(void *)) == 0)
+        return BCAST_OK;
+    const int rc = validate_bufs(rank_bufs, P, p.nbytes);
+    if (rc) return rc;
     ds.checked_bufs.assign(rank_bufs, rank_bufs + P);
     return BCAST_OK;
 }
@@ -426,18 +454,26 @@ void fill_ptrs(RankPtrs<MAXP> &rp, void *const *rank_bufs, int P)
 }
 
 template <int MAXP>
-int launch_walk(const bcast_device_state &ds, void *const *rank_bufs, int P, cudaStream_t st)
+int launch_walk_tables(int u, int grid, void *const *rank_bufs, int P, const WalkItem *items, int n_items,
+                       const uint32_t *hops, const int *hop_begin, WalkCtl *ctl, cudaStream_t st)
 {
     RankPtrs<MAXP> rp;
     fill_ptrs(rp, rank_bufs, P);
-    switch (ds.walk_u) {
-    case 8: bcast_walk_kernel<8, MAXP><<<ds.walk_grid, kThreads, 0, st>>>(rp, ds.d_items, ds.n_items, ds.d_hops, ds.d_hop_begin, ds.d_ctl); break;
-    case 4: bcast_walk_kernel<4, MAXP><<<ds.walk_grid, kThreads, 0, st>>>(rp, ds.d_items, ds.n_items, ds.d_hops, ds.d_hop_begin, ds.d_ctl); break;
-    case 2: bcast_walk_kernel<2, MAXP><<<ds.walk_grid, kThreads, 0, st>>>(rp, ds.d_items, ds.n_items, ds.d_hops, ds.d_hop_begin, ds.d_ctl); break;
-    default: bcast_walk_kernel<1, MAXP><<<ds.walk_grid, kThreads, 0, st>>>(rp, ds.d_items, ds.n_items, ds.d_hops, ds.d_hop_begin, ds.d_ctl); break;
+    switch (u) {
+    case 8: bcast_walk_kernel<8, MAXP><<<grid, kThreads, 0, st>>>(rp, items, n_items, hops, hop_begin, ctl); break;
+    case 4: bcast_walk_kernel<4, MAXP><<<grid, kThreads, 0, st>>>(rp, items, n_items, hops, hop_begin, ctl); break;
+    case 2: bcast_walk_kernel<2, MAXP><<<grid, kThreads, 0, st>>>(rp, items, n_items, hops, hop_begin, ctl); break;
+    default: bcast_walk_kernel<1, MAXP><<<grid, kThreads, 0, st>>>(rp, items, n_items, hops, hop_begin, ctl); break;
     }
     CUDA_TRY(cudaGetLastError());
     return BCAST_OK;
+}
+
+template <int MAXP>
+int launch_walk(const bcast_device_state &ds, void *const *rank_bufs, int P, cudaStream_t st)
+{
+    return launch_walk_tables<MAXP>(ds.walk_u, ds.walk_grid, rank_bufs, P, ds.d_items, ds.n_items, ds.d_hops,
+                                    ds.d_hop_begin, ds.d_ctl, st);
 }
 
 template <int MAXP>
@@ -566,3 +602,94 @@ int64_t bcast_exec_num_launches(const bcast_plan_t *plan, int mode)
 int bcast_last_cuda_error(void) { return t_last_cuda_error; }
 
 }  // extern "C"
+
+// ============================================================== execution without allocation
+// Scratch of bcast_exec_static(): lives in the library's device image, one copy per GPU that
+// loads it.  In host code this name is only a handle; the device address comes from
+// cudaGetSymbolAddress (once per device) and is what the kernel receives.
+static __device__ __align__(256) unsigned char g_static_scratch[BCAST_STATIC_SCRATCH_BYTES];
+
+namespace {
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mu;
+unsigned char *g_static_addr[kMaxDevices] = {};   // device address of g_static_scratch, per device
+int g_static_sms[kMaxDevices] = {};
+
+inline size_t round256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+// Device address of the scratch on the current device; looked up on the first call per device.
+int static_scratch(unsigned char **addr, int *sm_count)
+{
+    int device = -1;
+    CUDA_TRY(cudaGetDevice(&device));
+    if (device < 0 || device >= kMaxDevices) return BCAST_ERR_INVAL;
+    std::lock_guard<std::mutex> lock(g_static_mu);
+    if (!g_static_addr[device]) {
+        void *p = nullptr;
+        CUDA_TRY(cudaGetSymbolAddress(&p, g_static_scratch));
+        int sms = 0;
+        CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device));
+        g_static_addr[device] = (unsigned char *)p;
+        g_static_sms[device] = sms;
+    }
+    *addr = g_static_addr[device];
+    *sm_count = g_static_sms[device];
+    return BCAST_OK;
+}
+
+int exec_static(void *const *rank_bufs, const bcast_plan_t &p, cudaStream_t st)
+{
+    int rc = validate_bufs(rank_bufs, (size_t)p.P, p.nbytes);
+    if (rc) return rc;
+    if (p.total_bytes == 0) return BCAST_OK;
+    unsigned char *scratch = nullptr;
+    int sms = 0;
+    if ((rc = static_scratch(&scratch, &sms))) return rc;
+
+    // tables on the host; if they do not fit, try the largest tile before giving up
+    WalkTables t;
+    int u = choose_walk_words(p.nbytes, sms);
+    size_t off_hop_begin = 0, off_items = 0, off_hops = 0, total = 0;
+    for (;;) {
+        if ((rc = make_walk_tables(p, u, t))) return rc;
+        off_hop_begin = round256(sizeof(WalkCtl));
+        off_items = off_hop_begin + round256(t.hop_begin.size() * sizeof(int));
+        off_hops = off_items + round256(t.items.size() * sizeof(WalkItem));
+        total = off_hops + round256(t.hops.size() * sizeof(uint32_t));
+        if (total <= BCAST_STATIC_SCRATCH_BYTES) break;
+        if (u == 8) return BCAST_ERR_CAPACITY;
+        u = 8;
+    }
+    int bps = 1;
+    if ((rc = walk_blocks_per_sm(u, p.P, &bps))) return rc;
+    const int n_items = (int)t.items.size();
+    const int grid = std::max(1, std::min(n_items, sms * std::max(1, bps)));
+
+    // one image: zeroed work counter, then the three tables; a single stream-ordered copy puts it
+    // in place (the source is pageable host memory, which the runtime stages before returning)
+    std::vector<unsigned char> img(total, 0);
+    std::memcpy(img.data() + off_hop_begin, t.hop_begin.data(), t.hop_begin.size() * sizeof(int));
+    std::memcpy(img.data() + off_items, t.items.data(), t.items.size() * sizeof(WalkItem));
+    std::memcpy(img.data() + off_hops, t.hops.data(), t.hops.size() * sizeof(uint32_t));
+    CUDA_TRY(cudaMemcpyAsync(scratch, img.data(), total, cudaMemcpyHostToDevice, st));
+
+    WalkCtl *ctl = (WalkCtl *)scratch;
+    const int *hop_begin = (const int *)(scratch + off_hop_begin);
+    const WalkItem *items = (const WalkItem *)(scratch + off_items);
+    const uint32_t *hops = (const uint32_t *)(scratch + off_hops);
+    return p.P <= 128 ? launch_walk_tables<128>(u, grid, rank_bufs, p.P, items, n_items, hops, hop_begin, ctl, st)
+                      : launch_walk_tables<BCAST_MAX_RANKS>(u, grid, rank_bufs, p.P, items, n_items, hops, hop_begin, ctl, st);
+}
+
+}  // namespace
+
+extern "C" int bcast_exec_static(void *const *rank_bufs, const bcast_plan_t *plan, void *cuda_stream)
+{
+    if (!rank_bufs || !plan) return BCAST_ERR_INVAL;
+    try {
+        return exec_static(rank_bufs, *plan, (cudaStream_t)cuda_stream);
+    } catch (const std::bad_alloc &) {
+        return BCAST_ERR_NOMEM;
+    }
+}
