@@ -54,16 +54,23 @@ enum {
 /* How bcast_exec_mode() runs a plan.  All modes perform exactly the plan's messages. */
 enum {
     /* One launch for the whole plan.  The message is cut into tiles on a fixed grid of byte
-       offsets; a thread block takes a tile and carries it through every message of the plan
-       that covers it, in plan order (scatter hops first, then ring hops), re-reading it from
-       the source rank's buffer at every hop.  Messages that cover different byte ranges are
-       independent, so no cross-block waiting is needed.  Default of bcast_exec(). */
+       offsets; a warp takes a slice of a tile and carries it through every message of the plan
+       that covers it (scatter hops and ring hops), re-reading it from the source rank's buffer at
+       every hop.  Messages that cover different byte ranges are independent, so no waiting
+       between warps is needed.  The hops of a slice run in an order that respects every `dep`
+       of the plan (no copy is read before the message that delivers it has been performed) but
+       is not the plan's step order where a different order keeps the data in L2: see
+       BCAST_EXEC_WALK_PLAN_ORDER.  Default of bcast_exec(). */
     BCAST_EXEC_WALK = 0,
     /* One launch per plan step (ceil(log2 P) + P - 1 launches) on the caller's stream; inside a
        launch the messages of that step are cut into tiles and copied in parallel. */
     BCAST_EXEC_STEPS = 1,
     /* The same per-step launches, captured once into a CUDA graph and replayed. */
-    BCAST_EXEC_GRAPH = 2
+    BCAST_EXEC_GRAPH = 2,
+    /* BCAST_EXEC_WALK with the hops of every slice strictly in plan order (all scatter levels,
+       then the ring steps in ascending order).  Same copies, same result; in the tuned variant
+       the copies the scatter left at inner tree nodes are then re-read from DRAM instead of L2. */
+    BCAST_EXEC_WALK_PLAN_ORDER = 3
 };
 
 /* One message of the schedule.  Plain data, 48 bytes, host memory. */

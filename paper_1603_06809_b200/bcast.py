@@ -23,7 +23,7 @@ BCAST_NATIVE, BCAST_TUNED = 0, 1
 BCAST_PHASE_SCATTER, BCAST_PHASE_RING = 0, 1
 BCAST_OK, BCAST_ERR_INVAL, BCAST_ERR_NOMEM, BCAST_ERR_CUDA, BCAST_ERR_CAPACITY = 0, -1, -2, -3, -4
 BCAST_STATIC_SCRATCH_BYTES = 2 << 20
-BCAST_EXEC_WALK, BCAST_EXEC_STEPS, BCAST_EXEC_GRAPH = 0, 1, 2
+BCAST_EXEC_WALK, BCAST_EXEC_STEPS, BCAST_EXEC_GRAPH, BCAST_EXEC_WALK_PLAN_ORDER = 0, 1, 2, 3
 
 #: numpy view of ``bcast_xfer_t`` (48 bytes)
 XFER_DTYPE = np.dtype([

@@ -10,10 +10,10 @@
 //     from, so messages that cover different byte ranges never depend on one another.
 //
 // WALK executor (one launch): the message is cut into tiles on a fixed grid of byte offsets, split
-// further at chunk boundaries.  A thread block takes a tile and performs, in plan order, every
-// message that covers the tile's chunk, restricted to the tile: load from the source rank's
+// further at chunk boundaries.  A warp takes a slice of a tile and performs, in plan order, every
+// message that covers the tile's chunk, restricted to the slice: load from the source rank's
 // buffer, store to the destination rank's buffer.  Each thread always handles the same bytes of
-// the tile, so the load of hop h+1 reads what the same thread stored in hop h or earlier:
+// the slice, so the load of hop h+1 reads what the same thread stored in hop h or earlier:
 // program order per thread is the only ordering the schedule needs.  Loads bypass L1 (.cg) so that
 // every hop really re-reads the source rank's buffer from the L2/HBM level.
 //
@@ -34,7 +34,6 @@ namespace {
 constexpr int kThreads = 256;             // threads per block, both executors
 constexpr int kStepWordsPerThread = 4;    // STEPS executor: 256 x 4 x 16 B = 16 KiB tiles
 constexpr uint64_t kStepTile = (uint64_t)kThreads * kStepWordsPerThread * 16;
-constexpr int kMaxHops = BCAST_MAX_RANKS + 16;   // a chunk is covered by <= L + P - 1 messages
 
 thread_local int t_last_cuda_error = 0;
 
@@ -64,10 +63,6 @@ struct WalkItem {     // one tile of one chunk: bytes [lo, hi) of the message
     uint64_t lo, hi;
     int32_t chunk;    // relative chunk index: selects the hop list
     int32_t pad;
-};
-
-struct WalkCtl {      // work counter of the WALK executor; both fields are 0 between launches
-    unsigned int ticket, done;
 };
 
 // ---- memory operations.  volatile + "memory": the compiler must keep loads and stores of
@@ -115,73 +110,89 @@ __device__ __forceinline__ Split split16(uint64_t lo, uint64_t hi)
 }
 
 // ------------------------------------------------------------------------------------- WALK
+// A tile is 8 slices of 32 x U words; a warp owns one slice (U x 512 contiguous bytes) and walks
+// it through the chunk's hop list on its own: warps never wait for one another.  Slices are dealt
+// to warps round-robin (warp g takes slices g, g + G, ...), so the eight warps of a block work on
+// the eight slices of one tile and neighbouring blocks on neighbouring tiles.
+// The (src, dst) pair of hop h+1 is fetched while the loads of hop h are in flight.
+constexpr int kSlicesPerTile = kThreads / 32;
+
 template <int U, int MAXP>
 __global__ void __launch_bounds__(kThreads)
 bcast_walk_kernel(const __grid_constant__ RankPtrs<MAXP> bufs, const WalkItem *__restrict__ items, int n_items,
-                  const uint32_t *__restrict__ hops, const int *__restrict__ hop_begin, WalkCtl *ctl)
+                  const uint32_t *__restrict__ hops, const int *__restrict__ hop_begin)
 {
-    __shared__ uint32_t s_hops[kMaxHops];
-    __shared__ int s_item;
-    const int tid = threadIdx.x;
+    constexpr uint64_t kTile = (uint64_t)kThreads * U * 16;
+    const uint32_t lane = threadIdx.x & 31u;
+    const long long total_warps = (long long)gridDim.x * kSlicesPerTile;
+    const long long n_slices = (long long)n_items * kSlicesPerTile;
 
-    for (;;) {
-        if (tid == 0) s_item = (int)atomicAdd(&ctl->ticket, 1u);
-        __syncthreads();
-        const int it = s_item;
-        if (it >= n_items) break;
-        const WalkItem item = items[it];
-        const int hb = hop_begin[item.chunk];
-        const int nh = hop_begin[item.chunk + 1] - hb;
-        for (int h = tid; h < nh; h += kThreads) s_hops[h] = hops[hb + h];
-        __syncthreads();
+    for (long long w = (long long)blockIdx.x * kSlicesPerTile + (threadIdx.x >> 5); w < n_slices; w += total_warps) {
+        const WalkItem item = items[w / kSlicesPerTile];
+        const uint32_t slice = (uint32_t)(w % kSlicesPerTile);
+        // Words sit on the fixed 16-byte grid of the tile, whatever the chunk's first byte is, so
+        // that a warp's 512-byte accesses stay aligned to cache lines in ragged tiles too.
+        const uint64_t origin = item.lo / kTile * kTile + (uint64_t)slice * (32u * U * 16u);
+        const uint64_t body_lo = (item.lo + 15) & ~(uint64_t)15;     // first whole word of the item
+        const uint64_t body_hi = item.hi & ~(uint64_t)15;            // end of its last whole word
+        const uint64_t seg_lo = origin, seg_hi = origin + 32u * U * 16u;
+        // edge bytes (chunk start / end inside a word) belong to the slice that contains them
+        const uint64_t head_end = body_lo < item.hi ? body_lo : item.hi;
+        const uint64_t tail_begin = body_hi > head_end ? body_hi : head_end;
+        const uint32_t nhead = (item.lo >= seg_lo && item.lo < seg_hi) ? (uint32_t)(head_end - item.lo) : 0u;
+        const uint32_t ntail = (tail_begin >= seg_lo && tail_begin < seg_hi) ? (uint32_t)(item.hi - tail_begin) : 0u;
+        const uint32_t nedge = nhead + ntail;
+        const bool any_word = body_lo < body_hi && seg_lo < body_hi && body_lo < seg_hi;
+        if (!any_word && nedge == 0) continue;
+        const uint32_t *hp = hops + hop_begin[item.chunk];
+        const int nh = hop_begin[item.chunk + 1] - hop_begin[item.chunk];
+        const uint64_t base = origin + (uint64_t)lane * 16;
 
-        const Split sp = split16(item.lo, item.hi);
-        const uint64_t base = sp.a0 + (uint64_t)tid * 16;
-        if (sp.nwords == (uint32_t)(kThreads * U) && sp.nhead == 0 && sp.ntail == 0) {
-            // full tile: every thread moves U words per hop, no predicates
+        uint32_t e = __ldg(hp);
+        const uint8_t *s = bufs.p[e & 0xffffu];
+        uint8_t *d = bufs.p[e >> 16];
+        if (seg_lo >= body_lo && seg_hi <= body_hi && nedge == 0) {
+            // full slice: every lane moves U words per hop, no predicates
             for (int h = 0; h < nh; h++) {
-                const uint32_t e = s_hops[h];
-                const uint8_t *s = bufs.p[e & 0xffffu] + base;
-                uint8_t *d = bufs.p[e >> 16] + base;
                 uint4 v[U];
 #pragma unroll
-                for (int u = 0; u < U; u++) v[u] = ld16(s + (uint64_t)u * kThreads * 16);
+                for (int u = 0; u < U; u++) v[u] = ld16(s + base + (uint64_t)u * 512);
+                e = __ldg(hp + min(h + 1, nh - 1));              // next hop, while the loads are in flight
+                const uint8_t *s_next = bufs.p[e & 0xffffu];
+                uint8_t *d_next = bufs.p[e >> 16];
 #pragma unroll
-                for (int u = 0; u < U; u++) st16(d + (uint64_t)u * kThreads * 16, v[u]);
+                for (int u = 0; u < U; u++) st16(d + base + (uint64_t)u * 512, v[u]);
+                s = s_next;
+                d = d_next;
             }
         } else {
-            // ragged tile (chunk boundary or end of message): predicated words plus edge bytes,
-            // one byte per thread (at most 15 head + 15 tail bytes)
-            const uint32_t nedge = sp.nhead + sp.ntail;
-            const bool has_edge = (uint32_t)tid < nedge;
-            const uint64_t eoff = (uint32_t)tid < sp.nhead ? item.lo + tid : sp.tail_begin + (tid - sp.nhead);
+            // ragged slice (chunk boundary or end of message): predicated words, plus the <= 15 head
+            // and <= 15 tail bytes of the item, one byte per lane
+            bool ok[U];
+#pragma unroll
+            for (int u = 0; u < U; u++) {
+                const uint64_t o = base + (uint64_t)u * 512;
+                ok[u] = o >= body_lo && o + 16 <= body_hi;
+            }
+            const bool has_edge = lane < nedge;
+            const uint64_t eoff = lane < nhead ? item.lo + lane : tail_begin + (lane - nhead);
             for (int h = 0; h < nh; h++) {
-                const uint32_t e = s_hops[h];
-                const uint8_t *s = bufs.p[e & 0xffffu];
-                uint8_t *d = bufs.p[e >> 16];
                 uint4 v[U];
                 uint32_t b = 0;
 #pragma unroll
                 for (int u = 0; u < U; u++)
-                    if ((uint32_t)(tid + u * kThreads) < sp.nwords) v[u] = ld16(s + base + (uint64_t)u * kThreads * 16);
+                    if (ok[u]) v[u] = ld16(s + base + (uint64_t)u * 512);
                 if (has_edge) b = ld1(s + eoff);
+                e = __ldg(hp + min(h + 1, nh - 1));
+                const uint8_t *s_next = bufs.p[e & 0xffffu];
+                uint8_t *d_next = bufs.p[e >> 16];
 #pragma unroll
                 for (int u = 0; u < U; u++)
-                    if ((uint32_t)(tid + u * kThreads) < sp.nwords) st16(d + base + (uint64_t)u * kThreads * 16, v[u]);
+                    if (ok[u]) st16(d + base + (uint64_t)u * 512, v[u]);
                 if (has_edge) st1(d + eoff, b);
+                s = s_next;
+                d = d_next;
             }
-        }
-        __syncthreads();   // s_item and s_hops are rewritten by the next round
-    }
-
-    // the last block to leave puts the counters back to zero for the next launch
-    if (tid == 0) {
-        __threadfence();
-        const unsigned int d = atomicAdd(&ctl->done, 1u);
-        if (d == gridDim.x - 1) {
-            __threadfence();
-            ctl->ticket = 0;
-            ctl->done = 0;
         }
     }
 }
@@ -238,9 +249,9 @@ struct bcast_device_state {
     std::vector<void *> graph_bufs;
     // WALK
     WalkItem *d_items = nullptr;
-    uint32_t *d_hops = nullptr;
+    uint32_t *d_hops = nullptr;        // dependency order
+    uint32_t *d_hops_plan = nullptr;   // plan order
     int *d_hop_begin = nullptr;
-    WalkCtl *d_ctl = nullptr;
     int n_items = 0, walk_u = 0, walk_grid = 0;
     // argument check cache
     std::vector<void *> checked_bufs;
@@ -257,8 +268,8 @@ void bcast_device_state_free(bcast_device_state *dev)
     cudaFree(dev->d_xfers);
     cudaFree(dev->d_items);
     cudaFree(dev->d_hops);
+    cudaFree(dev->d_hops_plan);
     cudaFree(dev->d_hop_begin);
-    cudaFree(dev->d_ctl);
     if (switched) cudaSetDevice(cur);
     delete dev;
 }
@@ -316,9 +327,45 @@ int build_step_tables(const bcast_plan_t &p, bcast_device_state &ds)
 // and the tiles (fixed grid of `256 * u * 16`-byte offsets, split at chunk boundaries).
 struct WalkTables {
     std::vector<WalkItem> items;
-    std::vector<uint32_t> hops;
-    std::vector<int> hop_begin;   // [P + 1], by relative chunk index
+    std::vector<uint32_t> hops;        // per chunk, dependency order (see order_by_dependency)
+    std::vector<uint32_t> hops_plan;   // per chunk, plan order
+    std::vector<int> hop_begin;        // [P + 1], by relative chunk index; the same for both
 };
+
+// Re-order the hops of one chunk without breaking any dependency, so that a rank's copy is read
+// soon after it was written and is still in L2 then.
+//
+// In plan order the scatter hops come first and the ring hops later, so in the tuned ring every
+// copy that the scatter left at an inner node of the tree is read a second time ~P hops after it
+// was written, from DRAM.  The hops of a chunk form a tree: hop h hangs below the hop that wrote
+// its source rank (`dep` in the plan), or below the root's original data.  If no rank is written
+// twice, any order that puts a hop after its parent performs the same copies with the same result:
+// the data a hop reads is final once written.  The order chosen here is level order (breadth
+// first): all hops that read the same copy are neighbours, and the branches of the tree (the
+// ring segments that start at the root and at each inner node of the scatter tree) advance in
+// turn, so a copy is read again at most one level -- a handful of hops -- after it was written.
+// Chunks in which some rank is written more than once (native ring: redundant re-receives) keep
+// plan order, where write-after-read order matters.
+void order_by_dependency(const std::vector<uint32_t> &plan_order, int P, std::vector<uint32_t> &out)
+{
+    const int n = (int)plan_order.size();
+    out = plan_order;
+    std::vector<int> writer(P, -1);
+    for (int h = 0; h < n; h++) {
+        const int dst = (int)(plan_order[h] >> 16);
+        if (writer[dst] >= 0) return;                 // written twice: keep plan order
+        writer[dst] = h;
+    }
+    std::vector<int> depth(n), index(n);
+    for (int h = 0; h < n; h++) {
+        const int parent = writer[plan_order[h] & 0xffffu];
+        if (parent > h) return;                       // would read a copy before it exists: keep plan order
+        depth[h] = parent < 0 ? 0 : depth[parent] + 1;
+        index[h] = h;
+    }
+    std::stable_sort(index.begin(), index.end(), [&](int a, int b) { return depth[a] < depth[b]; });
+    for (int i = 0; i < n; i++) out[i] = plan_order[index[i]];
+}
 
 int make_walk_tables(const bcast_plan_t &p, int u, WalkTables &t)
 {
@@ -333,10 +380,13 @@ int make_walk_tables(const bcast_plan_t &p, int u, WalkTables &t)
     }
     t.hop_begin.assign(P + 1, 0);
     t.hops.clear();
+    t.hops_plan.clear();
+    std::vector<uint32_t> reordered;
     for (int c = 0; c < P; c++) {
-        if ((int)per_chunk[c].size() > kMaxHops) return BCAST_ERR_INVAL;
         t.hop_begin[c] = (int)t.hops.size();
-        t.hops.insert(t.hops.end(), per_chunk[c].begin(), per_chunk[c].end());
+        order_by_dependency(per_chunk[c], P, reordered);
+        t.hops.insert(t.hops.end(), reordered.begin(), reordered.end());
+        t.hops_plan.insert(t.hops_plan.end(), per_chunk[c].begin(), per_chunk[c].end());
     }
     t.hop_begin[P] = (int)t.hops.size();
 
@@ -363,6 +413,10 @@ int choose_walk_words(uint64_t nbytes, int sm_count)
     return 1;
 }
 
+// Resident blocks per SM the WALK executor aims for, by words per thread.  About 32 KB in flight
+// per SM saturates the memory system; more concurrent tiles only scatter the DRAM writes further.
+constexpr int kWalkBlocksPerSm(int u) { return u >= 4 ? 2 : u == 2 ? 3 : 8; }
+
 int walk_blocks_per_sm(int u, int P, int *bps)
 {
     if (P <= 128)
@@ -370,6 +424,23 @@ int walk_blocks_per_sm(int u, int P, int *bps)
              : u == 2 ? walk_occupancy<2, 128>(bps) : walk_occupancy<1, 128>(bps);
     return u == 8 ? walk_occupancy<8, BCAST_MAX_RANKS>(bps) : u == 4 ? walk_occupancy<4, BCAST_MAX_RANKS>(bps)
          : u == 2 ? walk_occupancy<2, BCAST_MAX_RANKS>(bps) : walk_occupancy<1, BCAST_MAX_RANKS>(bps);
+}
+
+// Blocks to launch: enough resident blocks per SM to keep the memory system busy, no more (see
+// kWalkBlocksPerSm), and never more blocks than tiles.
+int choose_walk_grid(int u, int P, int n_items, int sm_count, int *grid)
+{
+    int resident = 1;
+    const int rc = walk_blocks_per_sm(u, P, &resident);
+    if (rc) return rc;
+    const int want = env_int("BCAST_WALK_BLOCKS_PER_SM", kWalkBlocksPerSm(u));
+    const int most = std::max(1, std::min(n_items, sm_count * std::max(1, std::min(want, resident))));
+    // Every block takes tiles round-robin, so it runs ceil(n_items / grid) rounds.  Launch the
+    // fewest blocks that still need that many rounds: all rounds are then (almost) full instead of
+    // a last round that keeps a fraction of the GPU busy at memory latency.
+    const int rounds = (n_items + most - 1) / most;
+    *grid = std::max(1, (n_items + rounds - 1) / std::max(1, rounds));
+    return BCAST_OK;
 }
 
 // Device tables of the WALK executor, cached in the plan's device state.
@@ -380,16 +451,12 @@ int build_walk_tables(const bcast_plan_t &p, bcast_device_state &ds)
     int rc = make_walk_tables(p, ds.walk_u, t);
     if (rc) return rc;
     ds.n_items = (int)t.items.size();
-    int bps = 1;
-    if ((rc = walk_blocks_per_sm(ds.walk_u, p.P, &bps))) return rc;
-    const int cap = env_int("BCAST_WALK_BLOCKS_PER_SM", bps);
-    ds.walk_grid = std::max(1, std::min(ds.n_items, ds.sm_count * std::max(1, std::min(cap, bps))));
+    if ((rc = choose_walk_grid(ds.walk_u, p.P, ds.n_items, ds.sm_count, &ds.walk_grid))) return rc;
 
     if ((rc = upload(&ds.d_items, t.items))) return rc;
     if ((rc = upload(&ds.d_hops, t.hops))) return rc;
+    if ((rc = upload(&ds.d_hops_plan, t.hops_plan))) return rc;
     if ((rc = upload(&ds.d_hop_begin, t.hop_begin))) return rc;
-    CUDA_TRY(cudaMalloc((void **)&ds.d_ctl, sizeof(WalkCtl)));
-    CUDA_TRY(cudaMemset(ds.d_ctl, 0, sizeof(WalkCtl)));
     return BCAST_OK;
 }
 
@@ -455,25 +522,26 @@ void fill_ptrs(RankPtrs<MAXP> &rp, void *const *rank_bufs, int P)
 
 template <int MAXP>
 int launch_walk_tables(int u, int grid, void *const *rank_bufs, int P, const WalkItem *items, int n_items,
-                       const uint32_t *hops, const int *hop_begin, WalkCtl *ctl, cudaStream_t st)
+                       const uint32_t *hops, const int *hop_begin, cudaStream_t st)
 {
     RankPtrs<MAXP> rp;
     fill_ptrs(rp, rank_bufs, P);
     switch (u) {
-    case 8: bcast_walk_kernel<8, MAXP><<<grid, kThreads, 0, st>>>(rp, items, n_items, hops, hop_begin, ctl); break;
-    case 4: bcast_walk_kernel<4, MAXP><<<grid, kThreads, 0, st>>>(rp, items, n_items, hops, hop_begin, ctl); break;
-    case 2: bcast_walk_kernel<2, MAXP><<<grid, kThreads, 0, st>>>(rp, items, n_items, hops, hop_begin, ctl); break;
-    default: bcast_walk_kernel<1, MAXP><<<grid, kThreads, 0, st>>>(rp, items, n_items, hops, hop_begin, ctl); break;
+    case 8: bcast_walk_kernel<8, MAXP><<<grid, kThreads, 0, st>>>(rp, items, n_items, hops, hop_begin); break;
+    case 4: bcast_walk_kernel<4, MAXP><<<grid, kThreads, 0, st>>>(rp, items, n_items, hops, hop_begin); break;
+    case 2: bcast_walk_kernel<2, MAXP><<<grid, kThreads, 0, st>>>(rp, items, n_items, hops, hop_begin); break;
+    default: bcast_walk_kernel<1, MAXP><<<grid, kThreads, 0, st>>>(rp, items, n_items, hops, hop_begin); break;
     }
     CUDA_TRY(cudaGetLastError());
     return BCAST_OK;
 }
 
 template <int MAXP>
-int launch_walk(const bcast_device_state &ds, void *const *rank_bufs, int P, cudaStream_t st)
+int launch_walk(const bcast_device_state &ds, void *const *rank_bufs, int P, bool plan_order, cudaStream_t st)
 {
-    return launch_walk_tables<MAXP>(ds.walk_u, ds.walk_grid, rank_bufs, P, ds.d_items, ds.n_items, ds.d_hops,
-                                    ds.d_hop_begin, ds.d_ctl, st);
+    return launch_walk_tables<MAXP>(ds.walk_u, ds.walk_grid, rank_bufs, P, ds.d_items, ds.n_items,
+                                    plan_order ? ds.d_hops_plan : ds.d_hops,
+                                    ds.d_hop_begin, st);
 }
 
 template <int MAXP>
@@ -521,7 +589,9 @@ extern "C" {
 int bcast_exec_mode(void *const *rank_bufs, const bcast_plan_t *plan, void *cuda_stream, int mode)
 {
     if (!rank_bufs || !plan) return BCAST_ERR_INVAL;
-    if (mode != BCAST_EXEC_WALK && mode != BCAST_EXEC_STEPS && mode != BCAST_EXEC_GRAPH) return BCAST_ERR_INVAL;
+    if (mode != BCAST_EXEC_WALK && mode != BCAST_EXEC_STEPS && mode != BCAST_EXEC_GRAPH &&
+        mode != BCAST_EXEC_WALK_PLAN_ORDER)
+        return BCAST_ERR_INVAL;
     const bcast_plan_t &p = *plan;
     bcast_device_state *ds = nullptr;
     int rc = get_state(p, &ds);
@@ -537,7 +607,11 @@ int bcast_exec_mode(void *const *rank_bufs, const bcast_plan_t *plan, void *cuda
     const int P = p.P;
     switch (mode) {
     case BCAST_EXEC_WALK:
-        return P <= 128 ? launch_walk<128>(*ds, rank_bufs, P, st) : launch_walk<BCAST_MAX_RANKS>(*ds, rank_bufs, P, st);
+    case BCAST_EXEC_WALK_PLAN_ORDER: {
+        const bool plan_order = mode == BCAST_EXEC_WALK_PLAN_ORDER;
+        return P <= 128 ? launch_walk<128>(*ds, rank_bufs, P, plan_order, st)
+                        : launch_walk<BCAST_MAX_RANKS>(*ds, rank_bufs, P, plan_order, st);
+    }
     case BCAST_EXEC_STEPS:
         return P <= 128 ? launch_steps<128>(*ds, rank_bufs, P, st) : launch_steps<BCAST_MAX_RANKS>(*ds, rank_bufs, P, st);
     default:
@@ -586,7 +660,7 @@ int bcast_exec_host(void *const *rank_bufs, const bcast_plan_t *plan, void *cuda
 int64_t bcast_exec_num_launches(const bcast_plan_t *plan, int mode)
 {
     if (!plan || plan->total_bytes == 0) return 0;
-    if (mode == BCAST_EXEC_WALK) return 1;
+    if (mode == BCAST_EXEC_WALK || mode == BCAST_EXEC_WALK_PLAN_ORDER) return 1;
     if (mode != BCAST_EXEC_STEPS && mode != BCAST_EXEC_GRAPH) return 0;
     // a step launches a kernel unless all of its messages are empty
     int64_t n = 0;
@@ -653,7 +727,7 @@ int exec_static(void *const *rank_bufs, const bcast_plan_t &p, cudaStream_t st)
     size_t off_hop_begin = 0, off_items = 0, off_hops = 0, total = 0;
     for (;;) {
         if ((rc = make_walk_tables(p, u, t))) return rc;
-        off_hop_begin = round256(sizeof(WalkCtl));
+        off_hop_begin = 0;
         off_items = off_hop_begin + round256(t.hop_begin.size() * sizeof(int));
         off_hops = off_items + round256(t.items.size() * sizeof(WalkItem));
         total = off_hops + round256(t.hops.size() * sizeof(uint32_t));
@@ -661,25 +735,24 @@ int exec_static(void *const *rank_bufs, const bcast_plan_t &p, cudaStream_t st)
         if (u == 8) return BCAST_ERR_CAPACITY;
         u = 8;
     }
-    int bps = 1;
-    if ((rc = walk_blocks_per_sm(u, p.P, &bps))) return rc;
     const int n_items = (int)t.items.size();
-    const int grid = std::max(1, std::min(n_items, sms * std::max(1, bps)));
+    int grid = 1;
+    if ((rc = choose_walk_grid(u, p.P, n_items, sms, &grid))) return rc;
 
-    // one image: zeroed work counter, then the three tables; a single stream-ordered copy puts it
-    // in place (the source is pageable host memory, which the runtime stages before returning)
+    // one image of the three tables; a single stream-ordered copy puts it in place (the source is
+    // pageable host memory, which the runtime stages before returning).  Nothing in the array has
+    // to start at zero: the kernel only reads it.
     std::vector<unsigned char> img(total, 0);
     std::memcpy(img.data() + off_hop_begin, t.hop_begin.data(), t.hop_begin.size() * sizeof(int));
     std::memcpy(img.data() + off_items, t.items.data(), t.items.size() * sizeof(WalkItem));
     std::memcpy(img.data() + off_hops, t.hops.data(), t.hops.size() * sizeof(uint32_t));
     CUDA_TRY(cudaMemcpyAsync(scratch, img.data(), total, cudaMemcpyHostToDevice, st));
 
-    WalkCtl *ctl = (WalkCtl *)scratch;
     const int *hop_begin = (const int *)(scratch + off_hop_begin);
     const WalkItem *items = (const WalkItem *)(scratch + off_items);
     const uint32_t *hops = (const uint32_t *)(scratch + off_hops);
-    return p.P <= 128 ? launch_walk_tables<128>(u, grid, rank_bufs, p.P, items, n_items, hops, hop_begin, ctl, st)
-                      : launch_walk_tables<BCAST_MAX_RANKS>(u, grid, rank_bufs, p.P, items, n_items, hops, hop_begin, ctl, st);
+    return p.P <= 128 ? launch_walk_tables<128>(u, grid, rank_bufs, p.P, items, n_items, hops, hop_begin, st)
+                      : launch_walk_tables<BCAST_MAX_RANKS>(u, grid, rank_bufs, p.P, items, n_items, hops, hop_begin, st);
 }
 
 }  // namespace

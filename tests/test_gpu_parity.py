@@ -15,8 +15,8 @@ from gpu_harness import RankBuffers, run_broadcast
 
 pytestmark = pytest.mark.gpu
 
-MODES = [B.BCAST_EXEC_WALK, B.BCAST_EXEC_STEPS, B.BCAST_EXEC_GRAPH]
-MODE_IDS = ["walk", "steps", "graph"]
+MODES = [B.BCAST_EXEC_WALK, B.BCAST_EXEC_STEPS, B.BCAST_EXEC_GRAPH, B.BCAST_EXEC_WALK_PLAN_ORDER]
+MODE_IDS = ["walk", "steps", "graph", "walk_plan_order"]
 VARIANTS = [B.BCAST_NATIVE, B.BCAST_TUNED]
 VARIANT_IDS = ["native", "tuned"]
 
