@@ -24,8 +24,10 @@
  *   - "host" / "device" is stated for every pointer.  Ranks are ABSOLUTE ranks 0..P-1 unless a
  *     field says "relative" (relative rank r = (rank - root + P) mod P, Section IV listing).
  *   - A plan is immutable once created.  It may be executed any number of times; executions of
- *     the same plan must not overlap in time on the GPU (the plan caches small device-side
- *     tables and a work counter that executions share).
+ *     the same plan may overlap on the GPU if they use different rank buffers (the device-side
+ *     tables a plan caches are only read), except in BCAST_EXEC_GRAPH mode, whose captured graph
+ *     is bound to one set of buffers at a time.  The first execution of a plan (which builds those
+ *     tables) must not race with another call on the same plan.
  *   - The library keeps no other global state.  There is no CPU fallback: without a CUDA device
  *     the bcast_exec* calls fail with BCAST_ERR_CUDA.
  */
@@ -192,8 +194,8 @@ int bcast_exec_host(void *const *rank_bufs, const bcast_plan_t *plan, void *cuda
  *     512 MiB fit; P = 1024 does not.
  *   - The first call on a device looks up the array's device address (cudaGetSymbolAddress) and
  *     remembers it; make that first call outside any stream capture.
- *   - Every call re-writes the array (stream-ordered on cuda_stream) from host memory, including
- *     the work counter that has to start at zero, so the array's previous contents never matter.
+ *   - Every call re-writes the array (stream-ordered on cuda_stream) from host memory, so its
+ *     previous contents never matter; nothing in it has to start at zero (the kernel only reads it).
  *     Because all calls share the one array, two calls whose GPU work overlaps in time (different
  *     streams, or different host threads) race on it: serialise them.
  *   - No cudaMalloc, cudaFree or other allocating CUDA call is made; ordinary host heap memory is
@@ -202,6 +204,20 @@ int bcast_exec_host(void *const *rank_bufs, const bcast_plan_t *plan, void *cuda
  */
 #define BCAST_STATIC_SCRATCH_BYTES (2u << 20)
 int bcast_exec_static(void *const *rank_bufs, const bcast_plan_t *plan, void *cuda_stream);
+
+/*
+ * bcast_plan_walk_order -- the order in which BCAST_EXEC_WALK (or BCAST_EXEC_WALK_PLAN_ORDER)
+ * performs the messages that move bytes of one chunk.  Host only; needs no GPU.
+ *   chunk   relative chunk index 0..P-1
+ *   mode    BCAST_EXEC_WALK or BCAST_EXEC_WALK_PLAN_ORDER
+ *   out     HOST array of cap entries (may be NULL if cap = 0); receives indices into
+ *           bcast_plan_xfers(): every message with len > 0 whose chunk range contains `chunk` and
+ *           whose part of it is non-empty, each exactly once
+ * Returns the number of such messages (also when it exceeds cap; then only cap are written) or a
+ * negative BCAST_ERR_* code.  In both modes a message comes after the message named by its `dep`
+ * (Sections III-A and IV: a process can only pass on what it has received).
+ */
+int64_t bcast_plan_walk_order(const bcast_plan_t *plan, int chunk, int mode, int64_t *out, int64_t cap);
 
 /* Number of kernel launches one execution of the plan enqueues in the given mode (0 if nothing
    has to move); a CUDA-graph replay counts the kernels inside the graph. */

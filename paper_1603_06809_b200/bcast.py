@@ -36,7 +36,7 @@ SYMBOLS = (
     "bcast_plan", "bcast_plan_free", "bcast_plan_num_ranks", "bcast_plan_root", "bcast_plan_variant",
     "bcast_plan_nbytes", "bcast_plan_scatter_size", "bcast_plan_num_xfers", "bcast_plan_num_steps",
     "bcast_plan_xfers", "bcast_plan_step_begin", "bcast_plan_bytes_sent", "bcast_plan_bytes_recv",
-    "bcast_plan_msgs_sent", "bcast_plan_msgs_recv", "bcast_plan_total_bytes", "bcast_exec",
+    "bcast_plan_msgs_sent", "bcast_plan_msgs_recv", "bcast_plan_total_bytes", "bcast_plan_walk_order", "bcast_exec",
     "bcast_exec_mode", "bcast_exec_host", "bcast_exec_static", "bcast_exec_num_launches", "bcast_strerror",
     "bcast_last_cuda_error",
 )
@@ -53,6 +53,7 @@ _sig = {
     "bcast_plan_bytes_sent": (_vp, [_vp, _i]), "bcast_plan_bytes_recv": (_vp, [_vp, _i]),
     "bcast_plan_msgs_sent": (_vp, [_vp, _i]), "bcast_plan_msgs_recv": (_vp, [_vp, _i]),
     "bcast_plan_total_bytes": (_u64, [_vp]),
+    "bcast_plan_walk_order": (_i64, [_vp, _i, _i, ctypes.POINTER(ctypes.c_int64), _i64]),
     "bcast_exec": (_i, [_vpp, _vp, _vp]),
     "bcast_exec_mode": (_i, [_vpp, _vp, _vp, _i]),
     "bcast_exec_host": (_i, [_vpp, _vp, _vp, _i, _vp, _vpp]),
@@ -153,6 +154,20 @@ def bcast_plan_bytes_sent(plan: Plan, phase: int) -> np.ndarray: return _counter
 def bcast_plan_bytes_recv(plan: Plan, phase: int) -> np.ndarray: return _counter(_lib.bcast_plan_bytes_recv, plan, phase)
 def bcast_plan_msgs_sent(plan: Plan, phase: int) -> np.ndarray: return _counter(_lib.bcast_plan_msgs_sent, plan, phase)
 def bcast_plan_msgs_recv(plan: Plan, phase: int) -> np.ndarray: return _counter(_lib.bcast_plan_msgs_recv, plan, phase)
+
+
+def bcast_plan_walk_order(plan: Plan, chunk: int, mode: int = BCAST_EXEC_WALK) -> np.ndarray:
+    """Indices into the schedule of the messages that move chunk ``chunk``, in the order the WALK
+    executor performs them."""
+    n = _lib.bcast_plan_walk_order(plan.handle, chunk, mode, None, 0)
+    if n < 0:
+        raise BcastError(int(n), "bcast_plan_walk_order")
+    out = np.zeros(int(n), dtype=np.int64)
+    if n:
+        got = _lib.bcast_plan_walk_order(plan.handle, chunk, mode,
+                                         out.ctypes.data_as(ctypes.POINTER(ctypes.c_int64)), int(n))
+        assert got == n
+    return out
 
 
 def _ptr_array(items, what: str):

@@ -59,10 +59,9 @@ struct DevXfer {      // one message, device copy
     uint32_t pad;
 };
 
-struct WalkItem {     // one tile of one chunk: bytes [lo, hi) of the message
-    uint64_t lo, hi;
-    int32_t chunk;    // relative chunk index: selects the hop list
-    int32_t pad;
+struct WalkSlice {    // one warp's share of the message: segment `seg` of the fixed grid of
+    uint32_t seg;     // 32 * U * 16-byte segments, cut down to the bytes of relative chunk `chunk`
+    uint32_t chunk;   // (selects the hop list)
 };
 
 // ---- memory operations.  volatile + "memory": the compiler must keep loads and stores of
@@ -110,49 +109,42 @@ __device__ __forceinline__ Split split16(uint64_t lo, uint64_t hi)
 }
 
 // ------------------------------------------------------------------------------------- WALK
-// A tile is 8 slices of 32 x U words; a warp owns one slice (U x 512 contiguous bytes) and walks
-// it through the chunk's hop list on its own: warps never wait for one another.  Slices are dealt
-// to warps round-robin (warp g takes slices g, g + G, ...), so the eight warps of a block work on
-// the eight slices of one tile and neighbouring blocks on neighbouring tiles.
+// The message is cut on a fixed grid of segments of 32 x U words (U x 512 bytes), and every
+// segment further at chunk boundaries: a slice is the part of one segment that lies in one chunk.
+// A warp owns a slice and walks it through the chunk's hop list on its own: warps never wait for
+// one another.  Slices are dealt round-robin (warp g takes slices g, g + G, ...), so neighbouring
+// warps work on neighbouring segments.  Lanes map to the fixed 16-byte words of the segment,
+// whatever the chunk's first byte is, so a warp's 512-byte accesses stay aligned to cache lines;
+// the <= 15 bytes before the first whole word and after the last one go one byte per lane.
 // The (src, dst) pair of hop h+1 is fetched while the loads of hop h are in flight.
-constexpr int kSlicesPerTile = kThreads / 32;
+constexpr int kWarpsPerBlock = kThreads / 32;
 
 template <int U, int MAXP>
 __global__ void __launch_bounds__(kThreads)
-bcast_walk_kernel(const __grid_constant__ RankPtrs<MAXP> bufs, const WalkItem *__restrict__ items, int n_items,
+bcast_walk_kernel(const __grid_constant__ RankPtrs<MAXP> bufs, const WalkSlice *__restrict__ slices,
+                  long long n_slices, uint64_t scatter_size, uint64_t nbytes,
                   const uint32_t *__restrict__ hops, const int *__restrict__ hop_begin)
 {
-    constexpr uint64_t kTile = (uint64_t)kThreads * U * 16;
+    constexpr uint64_t kSeg = 32ull * U * 16;
     const uint32_t lane = threadIdx.x & 31u;
-    const long long total_warps = (long long)gridDim.x * kSlicesPerTile;
-    const long long n_slices = (long long)n_items * kSlicesPerTile;
+    const long long total_warps = (long long)gridDim.x * kWarpsPerBlock;
 
-    for (long long w = (long long)blockIdx.x * kSlicesPerTile + (threadIdx.x >> 5); w < n_slices; w += total_warps) {
-        const WalkItem item = items[w / kSlicesPerTile];
-        const uint32_t slice = (uint32_t)(w % kSlicesPerTile);
-        // Words sit on the fixed 16-byte grid of the tile, whatever the chunk's first byte is, so
-        // that a warp's 512-byte accesses stay aligned to cache lines in ragged tiles too.
-        const uint64_t origin = item.lo / kTile * kTile + (uint64_t)slice * (32u * U * 16u);
-        const uint64_t body_lo = (item.lo + 15) & ~(uint64_t)15;     // first whole word of the item
-        const uint64_t body_hi = item.hi & ~(uint64_t)15;            // end of its last whole word
-        const uint64_t seg_lo = origin, seg_hi = origin + 32u * U * 16u;
-        // edge bytes (chunk start / end inside a word) belong to the slice that contains them
-        const uint64_t head_end = body_lo < item.hi ? body_lo : item.hi;
-        const uint64_t tail_begin = body_hi > head_end ? body_hi : head_end;
-        const uint32_t nhead = (item.lo >= seg_lo && item.lo < seg_hi) ? (uint32_t)(head_end - item.lo) : 0u;
-        const uint32_t ntail = (tail_begin >= seg_lo && tail_begin < seg_hi) ? (uint32_t)(item.hi - tail_begin) : 0u;
-        const uint32_t nedge = nhead + ntail;
-        const bool any_word = body_lo < body_hi && seg_lo < body_hi && body_lo < seg_hi;
-        if (!any_word && nedge == 0) continue;
-        const uint32_t *hp = hops + hop_begin[item.chunk];
-        const int nh = hop_begin[item.chunk + 1] - hop_begin[item.chunk];
-        const uint64_t base = origin + (uint64_t)lane * 16;
+    for (long long w = (long long)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5); w < n_slices; w += total_warps) {
+        const WalkSlice sl = slices[w];
+        const uint64_t seg_lo = (uint64_t)sl.seg * kSeg, seg_hi = seg_lo + kSeg;
+        const uint64_t lo = max(min((uint64_t)sl.chunk * scatter_size, nbytes), seg_lo);
+        const uint64_t hi = min(min(((uint64_t)sl.chunk + 1) * scatter_size, nbytes), seg_hi);
+        if (lo >= hi) continue;
+        const uint32_t *hp = hops + hop_begin[sl.chunk];
+        const int nh = hop_begin[sl.chunk + 1] - hop_begin[sl.chunk];
+        if (nh <= 0) continue;
+        const uint64_t base = seg_lo + (uint64_t)lane * 16;
 
         uint32_t e = __ldg(hp);
         const uint8_t *s = bufs.p[e & 0xffffu];
         uint8_t *d = bufs.p[e >> 16];
-        if (seg_lo >= body_lo && seg_hi <= body_hi && nedge == 0) {
-            // full slice: every lane moves U words per hop, no predicates
+        if (lo == seg_lo && hi == seg_hi) {
+            // whole segment: every lane moves U words per hop, no predicates
             for (int h = 0; h < nh; h++) {
                 uint4 v[U];
 #pragma unroll
@@ -166,8 +158,12 @@ bcast_walk_kernel(const __grid_constant__ RankPtrs<MAXP> bufs, const WalkItem *_
                 d = d_next;
             }
         } else {
-            // ragged slice (chunk boundary or end of message): predicated words, plus the <= 15 head
-            // and <= 15 tail bytes of the item, one byte per lane
+            // ragged slice (a chunk starts or ends inside the segment): predicated words, plus the
+            // bytes of the partial words at either end
+            const uint64_t body_lo = (lo + 15) & ~(uint64_t)15, body_hi = hi & ~(uint64_t)15;
+            const uint64_t head_end = body_lo < hi ? body_lo : hi;
+            const uint64_t tail_begin = body_hi > head_end ? body_hi : head_end;
+            const uint32_t nhead = (uint32_t)(head_end - lo), nedge = nhead + (uint32_t)(hi - tail_begin);
             bool ok[U];
 #pragma unroll
             for (int u = 0; u < U; u++) {
@@ -175,7 +171,7 @@ bcast_walk_kernel(const __grid_constant__ RankPtrs<MAXP> bufs, const WalkItem *_
                 ok[u] = o >= body_lo && o + 16 <= body_hi;
             }
             const bool has_edge = lane < nedge;
-            const uint64_t eoff = lane < nhead ? item.lo + lane : tail_begin + (lane - nhead);
+            const uint64_t eoff = lane < nhead ? lo + lane : tail_begin + (lane - nhead);
             for (int h = 0; h < nh; h++) {
                 uint4 v[U];
                 uint32_t b = 0;
@@ -248,11 +244,12 @@ struct bcast_device_state {
     cudaGraphExec_t graph_exec = nullptr;
     std::vector<void *> graph_bufs;
     // WALK
-    WalkItem *d_items = nullptr;
+    WalkSlice *d_slices = nullptr;
     uint32_t *d_hops = nullptr;        // dependency order
     uint32_t *d_hops_plan = nullptr;   // plan order
     int *d_hop_begin = nullptr;
-    int n_items = 0, walk_u = 0, walk_grid = 0;
+    long long n_slices = 0;
+    int walk_u = 0, walk_grid = 0;
     // argument check cache
     std::vector<void *> checked_bufs;
 };
@@ -266,7 +263,7 @@ void bcast_device_state_free(bcast_device_state *dev)
     if (dev->graph_exec) cudaGraphExecDestroy(dev->graph_exec);
     if (dev->graph) cudaGraphDestroy(dev->graph);
     cudaFree(dev->d_xfers);
-    cudaFree(dev->d_items);
+    cudaFree(dev->d_slices);
     cudaFree(dev->d_hops);
     cudaFree(dev->d_hops_plan);
     cudaFree(dev->d_hop_begin);
@@ -326,7 +323,7 @@ int build_step_tables(const bcast_plan_t &p, bcast_device_state &ds)
 // Host form of the WALK executor's tables: per chunk the list of (src, dst) hops in plan order,
 // and the tiles (fixed grid of `256 * u * 16`-byte offsets, split at chunk boundaries).
 struct WalkTables {
-    std::vector<WalkItem> items;
+    std::vector<WalkSlice> slices;
     std::vector<uint32_t> hops;        // per chunk, dependency order (see order_by_dependency)
     std::vector<uint32_t> hops_plan;   // per chunk, plan order
     std::vector<int> hop_begin;        // [P + 1], by relative chunk index; the same for both
@@ -346,19 +343,19 @@ struct WalkTables {
 // turn, so a copy is read again at most one level -- a handful of hops -- after it was written.
 // Chunks in which some rank is written more than once (native ring: redundant re-receives) keep
 // plan order, where write-after-read order matters.
-void order_by_dependency(const std::vector<uint32_t> &plan_order, int P, std::vector<uint32_t> &out)
+void order_by_dependency(const bcast_plan_t &p, const std::vector<int64_t> &plan_order, std::vector<int64_t> &out)
 {
     const int n = (int)plan_order.size();
     out = plan_order;
-    std::vector<int> writer(P, -1);
+    std::vector<int> writer(p.P, -1);
     for (int h = 0; h < n; h++) {
-        const int dst = (int)(plan_order[h] >> 16);
+        const int dst = p.xfers[plan_order[h]].dst_rank;
         if (writer[dst] >= 0) return;                 // written twice: keep plan order
         writer[dst] = h;
     }
     std::vector<int> depth(n), index(n);
     for (int h = 0; h < n; h++) {
-        const int parent = writer[plan_order[h] & 0xffffu];
+        const int parent = writer[p.xfers[plan_order[h]].src_rank];
         if (parent > h) return;                       // would read a copy before it exists: keep plan order
         depth[h] = parent < 0 ? 0 : depth[parent] + 1;
         index[h] = h;
@@ -367,55 +364,60 @@ void order_by_dependency(const std::vector<uint32_t> &plan_order, int P, std::ve
     for (int i = 0; i < n; i++) out[i] = plan_order[index[i]];
 }
 
+// For every relative chunk: the plan's messages that move bytes of it, in plan order.
+void messages_by_chunk(const bcast_plan_t &p, std::vector<std::vector<int64_t>> &per_chunk)
+{
+    auto chunk_begin = [&](int c) { return std::min<uint64_t>((uint64_t)c * p.S, p.nbytes); };
+    per_chunk.assign(p.P, {});
+    for (size_t i = 0; i < p.xfers.size(); i++) {
+        const bcast_xfer_t &x = p.xfers[i];
+        if (!x.len) continue;
+        for (int c = x.chunk; c < x.chunk + x.nchunks; c++)
+            if (chunk_begin(c + 1) > chunk_begin(c)) per_chunk[c].push_back((int64_t)i);
+    }
+}
+
 int make_walk_tables(const bcast_plan_t &p, int u, WalkTables &t)
 {
     const int P = p.P;
     auto chunk_begin = [&](int c) { return std::min<uint64_t>((uint64_t)c * p.S, p.nbytes); };
-    std::vector<std::vector<uint32_t>> per_chunk(P);
-    for (const bcast_xfer_t &x : p.xfers) {
-        if (!x.len) continue;
-        const uint32_t e = (uint32_t)x.src_rank | ((uint32_t)x.dst_rank << 16);
-        for (int c = x.chunk; c < x.chunk + x.nchunks; c++)
-            if (chunk_begin(c + 1) > chunk_begin(c)) per_chunk[c].push_back(e);
-    }
+    auto encode = [&](int64_t i) { return (uint32_t)p.xfers[i].src_rank | ((uint32_t)p.xfers[i].dst_rank << 16); };
+    std::vector<std::vector<int64_t>> per_chunk;
+    messages_by_chunk(p, per_chunk);
     t.hop_begin.assign(P + 1, 0);
     t.hops.clear();
     t.hops_plan.clear();
-    std::vector<uint32_t> reordered;
+    std::vector<int64_t> reordered;
     for (int c = 0; c < P; c++) {
         t.hop_begin[c] = (int)t.hops.size();
-        order_by_dependency(per_chunk[c], P, reordered);
-        t.hops.insert(t.hops.end(), reordered.begin(), reordered.end());
-        t.hops_plan.insert(t.hops_plan.end(), per_chunk[c].begin(), per_chunk[c].end());
+        order_by_dependency(p, per_chunk[c], reordered);
+        for (int64_t i : reordered) t.hops.push_back(encode(i));
+        for (int64_t i : per_chunk[c]) t.hops_plan.push_back(encode(i));
     }
     t.hop_begin[P] = (int)t.hops.size();
 
-    const uint64_t tile = (uint64_t)kThreads * u * 16;
-    t.items.clear();
+    const uint64_t seg = 32ull * u * 16;
+    t.slices.clear();
     for (int c = 0; c < P; c++) {
         const uint64_t b = chunk_begin(c), e = chunk_begin(c + 1);
         if (e <= b || per_chunk[c].empty()) continue;
-        for (uint64_t g = b / tile; g * tile < e; g++)
-            t.items.push_back(WalkItem{std::max(b, g * tile), std::min(e, (g + 1) * tile), c, 0});
+        for (uint64_t g = b / seg; g * seg < e; g++) t.slices.push_back(WalkSlice{(uint32_t)g, (uint32_t)c});
     }
     return BCAST_OK;
 }
 
-// words per thread: large tiles when the message is big enough to fill the GPU with them
-int choose_walk_words(uint64_t nbytes, int sm_count)
+// Number of slices for U words per lane, without building the list.
+long long count_walk_slices(const bcast_plan_t &p, int u)
 {
-    const int forced = env_int("BCAST_WALK_WORDS", 0);
-    if (forced == 1 || forced == 2 || forced == 4 || forced == 8) return forced;
-    for (int cand : {4, 2}) {
-        const uint64_t tile = (uint64_t)kThreads * cand * 16;
-        if (nbytes / tile >= (uint64_t)sm_count * 8) return cand;
+    const uint64_t seg = 32ull * u * 16;
+    long long n = 0;
+    for (int c = 0; c < p.P; c++) {
+        const uint64_t b = std::min<uint64_t>((uint64_t)c * p.S, p.nbytes);
+        const uint64_t e = std::min<uint64_t>((uint64_t)(c + 1) * p.S, p.nbytes);
+        if (e > b) n += (long long)((e - 1) / seg - b / seg + 1);
     }
-    return 1;
+    return n;
 }
-
-// Resident blocks per SM the WALK executor aims for, by words per thread.  About 32 KB in flight
-// per SM saturates the memory system; more concurrent tiles only scatter the DRAM writes further.
-constexpr int kWalkBlocksPerSm(int u) { return u >= 4 ? 2 : u == 2 ? 3 : 8; }
 
 int walk_blocks_per_sm(int u, int P, int *bps)
 {
@@ -426,34 +428,73 @@ int walk_blocks_per_sm(int u, int P, int *bps)
          : u == 2 ? walk_occupancy<2, BCAST_MAX_RANKS>(bps) : walk_occupancy<1, BCAST_MAX_RANKS>(bps);
 }
 
-// Blocks to launch: enough resident blocks per SM to keep the memory system busy, no more (see
-// kWalkBlocksPerSm), and never more blocks than tiles.
-int choose_walk_grid(int u, int P, int n_items, int sm_count, int *grid)
+// Launch shape of the WALK executor: words per lane (U) and blocks.
+//   * Very few ranks (P <= 4): a slice makes at most three hops, the kernel is close to a plain
+//     copy and wants as many bytes in flight as the SMs can hold.
+//   * The whole message fits into the resident warps at once (one slice per warp): the run time is
+//     one walk down the longest hop list at memory latency, so take the smallest U that still fits
+//     -- the most warps, the fewest words each.
+//   * Otherwise the kernel is bound by the rate at which DRAM takes the scattered writes.  About
+//     32 KB in flight per SM (8 warps x 8 words x 512 B) saturate it; more concurrent slices only
+//     scatter the writes further.
+//     Every warp runs ceil(slices / warps) rounds; the fewest blocks that still need that many
+//     rounds are launched, so that all rounds are (almost) full instead of a last round that keeps
+//     a fraction of the GPU busy at memory latency.
+// BCAST_WALK_WORDS and BCAST_WALK_BLOCKS_PER_SM override the choice (for experiments).
+struct WalkShape {
+    int u = 1, grid = 1;
+};
+
+int choose_walk_shape(const bcast_plan_t &p, int sm_count, WalkShape *shape)
 {
-    int resident = 1;
-    const int rc = walk_blocks_per_sm(u, P, &resident);
-    if (rc) return rc;
-    const int want = env_int("BCAST_WALK_BLOCKS_PER_SM", kWalkBlocksPerSm(u));
-    const int most = std::max(1, std::min(n_items, sm_count * std::max(1, std::min(want, resident))));
-    // Every block takes tiles round-robin, so it runs ceil(n_items / grid) rounds.  Launch the
-    // fewest blocks that still need that many rounds: all rounds are then (almost) full instead of
-    // a last round that keeps a fraction of the GPU busy at memory latency.
-    const int rounds = (n_items + most - 1) / most;
-    *grid = std::max(1, (n_items + rounds - 1) / std::max(1, rounds));
+    const int forced_u = env_int("BCAST_WALK_WORDS", 0);
+    const int forced_bps = env_int("BCAST_WALK_BLOCKS_PER_SM", 0);
+    const bool u_ok = forced_u == 1 || forced_u == 2 || forced_u == 4 || forced_u == 8;
+    int rc, resident = 1, u = 0, bps = 0;
+    if (u_ok || forced_bps > 0) {
+        u = u_ok ? forced_u : 4;
+        if ((rc = walk_blocks_per_sm(u, p.P, &resident))) return rc;
+        bps = forced_bps > 0 ? std::min(forced_bps, resident) : resident;
+    } else if (p.P <= 4) {
+        u = 2;
+        if ((rc = walk_blocks_per_sm(u, p.P, &resident))) return rc;
+        bps = resident;
+    } else {
+        for (int cand : {1, 2, 4, 8}) {
+            if ((rc = walk_blocks_per_sm(cand, p.P, &resident))) return rc;
+            if (count_walk_slices(p, cand) <= (long long)sm_count * resident * kWarpsPerBlock) {
+                u = cand;
+                bps = resident;
+                break;
+            }
+        }
+        if (!u) {
+            // eight words per lane; one block per SM once that alone gives six or more rounds
+            u = 8;
+            bps = count_walk_slices(p, u) >= 6ll * sm_count * kWarpsPerBlock ? 1 : 2;
+        }
+    }
+    const long long slices = std::max<long long>(1, count_walk_slices(p, u));
+    const long long most = (long long)sm_count * std::max(1, bps) * kWarpsPerBlock;   // warps
+    const long long rounds = (slices + most - 1) / most;
+    const long long warps = (slices + rounds - 1) / rounds;
+    shape->u = u;
+    shape->grid = (int)std::max<long long>(1, (warps + kWarpsPerBlock - 1) / kWarpsPerBlock);
     return BCAST_OK;
 }
 
 // Device tables of the WALK executor, cached in the plan's device state.
 int build_walk_tables(const bcast_plan_t &p, bcast_device_state &ds)
 {
-    ds.walk_u = choose_walk_words(p.nbytes, ds.sm_count);
-    WalkTables t;
-    int rc = make_walk_tables(p, ds.walk_u, t);
+    WalkShape shape;
+    int rc = choose_walk_shape(p, ds.sm_count, &shape);
     if (rc) return rc;
-    ds.n_items = (int)t.items.size();
-    if ((rc = choose_walk_grid(ds.walk_u, p.P, ds.n_items, ds.sm_count, &ds.walk_grid))) return rc;
-
-    if ((rc = upload(&ds.d_items, t.items))) return rc;
+    ds.walk_u = shape.u;
+    ds.walk_grid = shape.grid;
+    WalkTables t;
+    if ((rc = make_walk_tables(p, ds.walk_u, t))) return rc;
+    ds.n_slices = (long long)t.slices.size();
+    if ((rc = upload(&ds.d_slices, t.slices))) return rc;
     if ((rc = upload(&ds.d_hops, t.hops))) return rc;
     if ((rc = upload(&ds.d_hops_plan, t.hops_plan))) return rc;
     if ((rc = upload(&ds.d_hop_begin, t.hop_begin))) return rc;
@@ -520,28 +561,41 @@ void fill_ptrs(RankPtrs<MAXP> &rp, void *const *rank_bufs, int P)
     for (int k = P; k < MAXP; k++) rp.p[k] = nullptr;
 }
 
+struct WalkLaunch {     // everything one WALK launch needs besides the rank pointers
+    int u, grid;
+    const WalkSlice *slices;
+    long long n_slices;
+    uint64_t scatter_size, nbytes;
+    const uint32_t *hops;
+    const int *hop_begin;
+};
+
 template <int MAXP>
-int launch_walk_tables(int u, int grid, void *const *rank_bufs, int P, const WalkItem *items, int n_items,
-                       const uint32_t *hops, const int *hop_begin, cudaStream_t st)
+int launch_walk_tables(const WalkLaunch &w, void *const *rank_bufs, int P, cudaStream_t st)
 {
     RankPtrs<MAXP> rp;
     fill_ptrs(rp, rank_bufs, P);
-    switch (u) {
-    case 8: bcast_walk_kernel<8, MAXP><<<grid, kThreads, 0, st>>>(rp, items, n_items, hops, hop_begin); break;
-    case 4: bcast_walk_kernel<4, MAXP><<<grid, kThreads, 0, st>>>(rp, items, n_items, hops, hop_begin); break;
-    case 2: bcast_walk_kernel<2, MAXP><<<grid, kThreads, 0, st>>>(rp, items, n_items, hops, hop_begin); break;
-    default: bcast_walk_kernel<1, MAXP><<<grid, kThreads, 0, st>>>(rp, items, n_items, hops, hop_begin); break;
+#define BCAST_WALK_LAUNCH(U_)                                                                       \
+    bcast_walk_kernel<U_, MAXP><<<w.grid, kThreads, 0, st>>>(rp, w.slices, w.n_slices, w.scatter_size, \
+                                                             w.nbytes, w.hops, w.hop_begin)
+    switch (w.u) {
+    case 8: BCAST_WALK_LAUNCH(8); break;
+    case 4: BCAST_WALK_LAUNCH(4); break;
+    case 2: BCAST_WALK_LAUNCH(2); break;
+    default: BCAST_WALK_LAUNCH(1); break;
     }
+#undef BCAST_WALK_LAUNCH
     CUDA_TRY(cudaGetLastError());
     return BCAST_OK;
 }
 
-template <int MAXP>
-int launch_walk(const bcast_device_state &ds, void *const *rank_bufs, int P, bool plan_order, cudaStream_t st)
+int launch_walk(const bcast_plan_t &p, const bcast_device_state &ds, void *const *rank_bufs, bool plan_order,
+                cudaStream_t st)
 {
-    return launch_walk_tables<MAXP>(ds.walk_u, ds.walk_grid, rank_bufs, P, ds.d_items, ds.n_items,
-                                    plan_order ? ds.d_hops_plan : ds.d_hops,
-                                    ds.d_hop_begin, st);
+    const WalkLaunch w{ds.walk_u, ds.walk_grid, ds.d_slices, ds.n_slices, p.S, p.nbytes,
+                       plan_order ? ds.d_hops_plan : ds.d_hops, ds.d_hop_begin};
+    return p.P <= 128 ? launch_walk_tables<128>(w, rank_bufs, p.P, st)
+                      : launch_walk_tables<BCAST_MAX_RANKS>(w, rank_bufs, p.P, st);
 }
 
 template <int MAXP>
@@ -608,9 +662,7 @@ int bcast_exec_mode(void *const *rank_bufs, const bcast_plan_t *plan, void *cuda
     switch (mode) {
     case BCAST_EXEC_WALK:
     case BCAST_EXEC_WALK_PLAN_ORDER: {
-        const bool plan_order = mode == BCAST_EXEC_WALK_PLAN_ORDER;
-        return P <= 128 ? launch_walk<128>(*ds, rank_bufs, P, plan_order, st)
-                        : launch_walk<BCAST_MAX_RANKS>(*ds, rank_bufs, P, plan_order, st);
+        return launch_walk(p, *ds, rank_bufs, mode == BCAST_EXEC_WALK_PLAN_ORDER, st);
     }
     case BCAST_EXEC_STEPS:
         return P <= 128 ? launch_steps<128>(*ds, rank_bufs, P, st) : launch_steps<BCAST_MAX_RANKS>(*ds, rank_bufs, P, st);
@@ -655,6 +707,22 @@ int bcast_exec_host(void *const *rank_bufs, const bcast_plan_t *plan, void *cuda
                 CUDA_TRY(cudaMemcpyAsync(host_out[k], rank_bufs[k], p.nbytes, cudaMemcpyDeviceToHost, st));
     CUDA_TRY(cudaStreamSynchronize(st));
     return BCAST_OK;
+}
+
+int64_t bcast_plan_walk_order(const bcast_plan_t *plan, int chunk, int mode, int64_t *out, int64_t cap)
+{
+    if (!plan || chunk < 0 || chunk >= plan->P || cap < 0 || (cap > 0 && !out)) return BCAST_ERR_INVAL;
+    if (mode != BCAST_EXEC_WALK && mode != BCAST_EXEC_WALK_PLAN_ORDER) return BCAST_ERR_INVAL;
+    try {
+        std::vector<std::vector<int64_t>> per_chunk;
+        messages_by_chunk(*plan, per_chunk);
+        std::vector<int64_t> order = per_chunk[chunk];
+        if (mode == BCAST_EXEC_WALK) order_by_dependency(*plan, per_chunk[chunk], order);
+        for (int64_t i = 0; i < (int64_t)order.size() && i < cap; i++) out[i] = order[i];
+        return (int64_t)order.size();
+    } catch (const std::bad_alloc &) {
+        return BCAST_ERR_NOMEM;
+    }
 }
 
 int64_t bcast_exec_num_launches(const bcast_plan_t *plan, int mode)
@@ -721,38 +789,35 @@ int exec_static(void *const *rank_bufs, const bcast_plan_t &p, cudaStream_t st)
     int sms = 0;
     if ((rc = static_scratch(&scratch, &sms))) return rc;
 
-    // tables on the host; if they do not fit, try the largest tile before giving up
+    // tables on the host; if they do not fit, try the largest slices before giving up
+    WalkShape shape;
+    if ((rc = choose_walk_shape(p, sms, &shape))) return rc;
     WalkTables t;
-    int u = choose_walk_words(p.nbytes, sms);
-    size_t off_hop_begin = 0, off_items = 0, off_hops = 0, total = 0;
+    size_t off_slices = 0, off_hops = 0, total = 0;
     for (;;) {
-        if ((rc = make_walk_tables(p, u, t))) return rc;
-        off_hop_begin = 0;
-        off_items = off_hop_begin + round256(t.hop_begin.size() * sizeof(int));
-        off_hops = off_items + round256(t.items.size() * sizeof(WalkItem));
+        if ((rc = make_walk_tables(p, shape.u, t))) return rc;
+        off_slices = round256(t.hop_begin.size() * sizeof(int));
+        off_hops = off_slices + round256(t.slices.size() * sizeof(WalkSlice));
         total = off_hops + round256(t.hops.size() * sizeof(uint32_t));
         if (total <= BCAST_STATIC_SCRATCH_BYTES) break;
-        if (u == 8) return BCAST_ERR_CAPACITY;
-        u = 8;
+        if (shape.u == 8) return BCAST_ERR_CAPACITY;
+        shape.u = 8;
+        shape.grid = std::max(1, std::min<int>(shape.grid, (int)((count_walk_slices(p, 8) + kWarpsPerBlock - 1) / kWarpsPerBlock)));
     }
-    const int n_items = (int)t.items.size();
-    int grid = 1;
-    if ((rc = choose_walk_grid(u, p.P, n_items, sms, &grid))) return rc;
 
     // one image of the three tables; a single stream-ordered copy puts it in place (the source is
     // pageable host memory, which the runtime stages before returning).  Nothing in the array has
     // to start at zero: the kernel only reads it.
     std::vector<unsigned char> img(total, 0);
-    std::memcpy(img.data() + off_hop_begin, t.hop_begin.data(), t.hop_begin.size() * sizeof(int));
-    std::memcpy(img.data() + off_items, t.items.data(), t.items.size() * sizeof(WalkItem));
+    std::memcpy(img.data(), t.hop_begin.data(), t.hop_begin.size() * sizeof(int));
+    std::memcpy(img.data() + off_slices, t.slices.data(), t.slices.size() * sizeof(WalkSlice));
     std::memcpy(img.data() + off_hops, t.hops.data(), t.hops.size() * sizeof(uint32_t));
     CUDA_TRY(cudaMemcpyAsync(scratch, img.data(), total, cudaMemcpyHostToDevice, st));
 
-    const int *hop_begin = (const int *)(scratch + off_hop_begin);
-    const WalkItem *items = (const WalkItem *)(scratch + off_items);
-    const uint32_t *hops = (const uint32_t *)(scratch + off_hops);
-    return p.P <= 128 ? launch_walk_tables<128>(u, grid, rank_bufs, p.P, items, n_items, hops, hop_begin, st)
-                      : launch_walk_tables<BCAST_MAX_RANKS>(u, grid, rank_bufs, p.P, items, n_items, hops, hop_begin, st);
+    const WalkLaunch w{shape.u, shape.grid, (const WalkSlice *)(scratch + off_slices), (long long)t.slices.size(),
+                       p.S, p.nbytes, (const uint32_t *)(scratch + off_hops), (const int *)scratch};
+    return p.P <= 128 ? launch_walk_tables<128>(w, rank_bufs, p.P, st)
+                      : launch_walk_tables<BCAST_MAX_RANKS>(w, rank_bufs, p.P, st);
 }
 
 }  // namespace

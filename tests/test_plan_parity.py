@@ -132,3 +132,68 @@ def test_exec_without_gpu_fails_loudly():
     with pytest.raises(B.BcastError) as e:
         B.bcast_exec([4096, 8192, 12288, 16384], plan)
     assert e.value.code == B.BCAST_ERR_CUDA
+
+
+@pytest.mark.parametrize("variant", [B.BCAST_NATIVE, B.BCAST_TUNED])
+def test_walk_order_respects_every_dependency(oracle, variant):
+    """The order in which the one-launch executor performs the messages of a chunk (both of its
+    modes): the same messages as the oracle's schedule has for that chunk, each once; a message
+    never before the message named by its `dep`; replayed in that order, the sender always holds
+    the chunk already and in the end every rank holds it."""
+    for P, root, n in [(2, 1, 64), (8, 0, 1 << 12), (10, 3, 12345), (12, 5, 256 << 10), (33, 32, 100003),
+                       (64, 17, (16 << 20) + 13), (100, 63, 64 << 20), (255, 254, 12288)]:
+        plan = B.bcast_plan(P, root, n, variant)
+        ref = oracle.simulate(P, root, n, variant)
+        S = ref.scatter_size
+        sched = ref.schedule
+        for c in sorted({0, 1, P // 2, P - 2, P - 1} & set(range(P))):
+            clen = min((c + 1) * S, n) - min(c * S, n)
+            want = [i for i in range(len(sched))
+                    if sched[i, 7] > 0 and sched[i, 4] <= c < sched[i, 4] + sched[i, 5] and clen > 0]
+            plan_order = B.bcast_plan_walk_order(plan, c, B.BCAST_EXEC_WALK_PLAN_ORDER)
+            walk_order = B.bcast_plan_walk_order(plan, c, B.BCAST_EXEC_WALK)
+            assert list(plan_order) == want
+            assert sorted(walk_order) == want
+            if variant == B.BCAST_NATIVE:
+                assert list(walk_order) == want          # ranks are re-written: plan order is kept
+            for order in (plan_order, walk_order):
+                pos = {int(m): k for k, m in enumerate(order)}
+                holders = {root}
+                for m in order:
+                    dep = int(sched[m, 8])
+                    if dep >= 0:
+                        assert dep in pos and pos[dep] < pos[int(m)]
+                    assert int(sched[m, 2]) in holders
+                    holders.add(int(sched[m, 3]))
+                if want:
+                    assert holders == set(range(P))
+    with pytest.raises(B.BcastError):
+        B.bcast_plan_walk_order(B.bcast_plan(4, 0, 64, 1), 4)
+    with pytest.raises(B.BcastError):
+        B.bcast_plan_walk_order(B.bcast_plan(4, 0, 64, 1), 0, B.BCAST_EXEC_STEPS)
+
+
+def test_walk_order_reads_follow_writes_closely():
+    """Tuned ring: in the one-launch executor's order a copy is read at most a few messages after
+    it was written (one level of the dependency tree), never ~P messages later as in plan order."""
+    P, root, n = 100, 63, 64 << 20
+    plan = B.bcast_plan(P, root, n, B.BCAST_TUNED)
+    x = B.bcast_plan_xfers(plan)
+    L = (P - 1).bit_length()
+    worst_walk, worst_plan = 0, 0
+    for c in range(P):
+        for mode in (B.BCAST_EXEC_WALK, B.BCAST_EXEC_WALK_PLAN_ORDER):
+            order = B.bcast_plan_walk_order(plan, c, mode)
+            written_at = {}
+            worst = 0
+            for k, m in enumerate(order):
+                src, dst = int(x[m]["src_rank"]), int(x[m]["dst_rank"])
+                if src in written_at:
+                    worst = max(worst, k - written_at[src])
+                written_at[dst] = k
+            if mode == B.BCAST_EXEC_WALK:
+                worst_walk = max(worst_walk, worst)
+            else:
+                worst_plan = max(worst_plan, worst)
+    assert worst_walk <= 2 * (L + 1)
+    assert worst_plan > P // 2
