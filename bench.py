@@ -38,15 +38,43 @@ FALLBACK_HBM_GBS = 6650.0
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg4", choices=["cfg3", "cfg4"])
     ap.add_argument("--mode", default="walk", choices=["walk", "walk_plan_order", "steps", "graph"])
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-clocks", action="store_true", help="skip the nvidia-smi sampling and its extra load (profiling runs)")
+    ap.add_argument("--no-clocks", action="store_true", help="skip the nvidia-smi sampling (profiling runs)")
     return ap.parse_args()
+
+
+# DRAM bytes of one launch of the dominant kernel (tuned variant), from ncu:
+# dram__bytes_read.sum + dram__bytes_write.sum.  A figure is only valid for the kernel source it
+# was taken with, so each carries the SHA-256 of csrc/exec.cu; once the file changes, `traffic`
+# is reported as null until the counters are taken again.
+NCU_TRAFFIC = {
+    # profiles/bcast_walk_kernel_P100_64MiB_launch_list_and_dram.md
+    ("cfg4", "walk"): {"dram_bytes_per_launch": 6.658e9,
+                       "exec_cu_sha256": "084fe303ec385a617f3d74dcdcd1ba494b6f1ac16bb06c1a8382149b4b7f48b0"},
+    # profiles/bcast_walk_kernel_P64_16MiB_ncu_full.md
+    ("cfg3", "walk"): {"dram_bytes_per_launch": 1.018e9,
+                       "exec_cu_sha256": "084fe303ec385a617f3d74dcdcd1ba494b6f1ac16bb06c1a8382149b4b7f48b0"},
+}
+
+
+def ncu_traffic(workload, mode):
+    import hashlib
+    rec = NCU_TRAFFIC.get((workload, mode))
+    if not rec:
+        return None
+    path = os.path.join(ROOT, "paper_1603_06809_b200", "csrc", "exec.cu")
+    try:
+        with open(path, "rb") as f:
+            sha = hashlib.sha256(f.read()).hexdigest()
+    except OSError:
+        return None
+    return rec["dram_bytes_per_launch"] if sha == rec["exec_cu_sha256"] else None
 
 
 def measured_peak():
@@ -60,9 +88,12 @@ def measured_peak():
 
 # --------------------------------------------------------------------------- clocks during the run
 class ClockSampler:
-    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+    """nvidia-smi in a loop while the benchmark runs; only samples whose timestamp falls inside
+    the timed region are used (the nearest ones if the region was too short to be hit)."""
+    QUERY = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    NAMES = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
 
     def __init__(self, gpu_index: int):
         self.gpu = gpu_index
@@ -76,12 +107,14 @@ class ClockSampler:
             self.out = open(self.path, "w")
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=self.out, stderr=subprocess.DEVNULL)
+                 "-lms", "20"], stdout=self.out, stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
 
-    def stop(self):
-        res = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+    def stop(self, t_begin: float, t_end: float):
+        """t_begin / t_end: time.time() at the two ends of the timed region."""
+        import datetime
+        res = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0, "power_w": None}
         if self.proc is None:
             return res
         self.proc.terminate()
@@ -90,8 +123,7 @@ class ClockSampler:
         except Exception:
             self.proc.kill()
         self.out.close()
-        sm, smax, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        rows = []
         try:
             with open(self.path) as f:
                 for line in f:
@@ -99,18 +131,24 @@ class ClockSampler:
                     if len(c) < 9:
                         continue
                     try:
-                        sm.append(float(c[1])); smax.append(float(c[2]))
+                        ts = datetime.datetime.strptime(c[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                        rows.append((ts, float(c[1]), float(c[2]), float(c[3]),
+                                     [n for n, v in zip(self.NAMES, c[5:9]) if v.lower().startswith("active")]))
                     except ValueError:
                         continue
-                    for name, val in zip(names, c[5:9]):
-                        if val.lower().startswith("active"):
-                            reasons.add(name)
             os.unlink(self.path)
         except Exception:
             pass
-        if sm:
-            res.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(smax), samples=len(sm))
-        res["reasons"] = sorted(reasons)
+        inside = [r for r in rows if t_begin <= r[0] <= t_end]
+        where = "inside the timed region"
+        if not inside and rows:
+            mid = 0.5 * (t_begin + t_end)
+            inside = sorted(rows, key=lambda r: abs(r[0] - mid))[:3]
+            where = "nearest to the timed region (it was shorter than the sampling interval)"
+        if inside:
+            res.update(sm_mhz=statistics.median(r[1] for r in inside), sm_max_mhz=max(r[2] for r in inside),
+                       power_w=round(statistics.median(r[3] for r in inside), 1), samples=len(inside), taken=where)
+            res["reasons"] = sorted({n for r in inside for n in r[4]})
         return res
 
 
@@ -153,36 +191,24 @@ def run_ours(args):
         torch.cuda.synchronize()
 
     def timed(plan, steps, warmup, sample_clocks=False):
-        """`steps` broadcasts between two events; also one event pair around every launch."""
+        """`steps` broadcasts between two events; also one event per launch."""
         sampler = ClockSampler(local_rank) if sample_clocks else None
         if sampler:
             sampler.start()
-
-        def load_for(seconds):
-            # untimed broadcasts, so that every clock sample is taken under the benchmark's own load
-            t_end = time.time() + seconds
-            while time.time() < t_end:
-                for _ in range(20):
-                    B.bcast_exec_mode(ptrs, plan, stream, mode)
-                torch.cuda.synchronize()
-
         for _ in range(warmup):
             B.bcast_exec_mode(ptrs, plan, stream, mode)
-        if sampler:
-            load_for(0.5)
         ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
         barrier()
+        t_begin = time.time()
         ev[0].record(stream)
         for i in range(steps):
             B.bcast_exec_mode(ptrs, plan, stream, mode)
             ev[i + 1].record(stream)
         barrier()
+        t_end = time.time()
         total_ms = ev[0].elapsed_time(ev[steps])
         per = [ev[i].elapsed_time(ev[i + 1]) for i in range(steps)]
-        clocks = None
-        if sampler:
-            load_for(0.5)
-            clocks = sampler.stop()
+        clocks = sampler.stop(t_begin, t_end) if sampler else None
         if world > 1:
             t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
             dist.all_reduce(t, op=dist.ReduceOp.MAX)
@@ -214,16 +240,7 @@ def run_ours(args):
     launch_ms = statistics.mean(tuned["per"]) / max(1, tuned["launches"])
     alg_bytes_per_launch = 2 * tuned["moved"] / max(1, tuned["launches"])
     achieved = alg_bytes_per_launch / (launch_ms * 1e-3) / 1e9
-    traffic = None
-    traffic_note = os.path.join(ROOT, "profiles", "dram_traffic.json")
-    try:
-        with open(traffic_note) as f:
-            tj = json.load(f)
-        key = f"{args.workload}_{args.mode}_tuned"
-        if key in tj:
-            traffic = tj[key]["dram_bytes_per_launch"]
-    except Exception:
-        pass
+    traffic = ncu_traffic(args.workload, args.mode)
     roofline = {
         "bound": "hbm", "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
         "frac": round(achieved / peak, 4), "traffic": traffic,
@@ -232,8 +249,9 @@ def run_ours(args):
         "algorithmic_bytes_per_launch": alg_bytes_per_launch,
         "launch_ms": round(launch_ms, 5),
         "frac_of_nominal_8TBps": round(achieved / NOMINAL_HBM_GBS, 4),
-        "note": "algorithmic bytes = read + write of every scheduled byte; re-reads of a tile by the hop "
-                "that follows its write are served by L2, so DRAM traffic is about half of this",
+        "note": "algorithmic bytes = read + write of every scheduled byte; the read of a hop hits in L2 on what "
+                "an earlier hop stored microseconds before, so DRAM sees about half of this (every rank "
+                "buffer written once, the root's message read once): frac > 1 is expected",
     }
 
     # ---- end to end through the host-buffer entry point: H2D of the message, broadcast, D2H of all P buffers
