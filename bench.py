@@ -152,6 +152,25 @@ class ClockSampler:
         return res
 
 
+# --------------------------------------------------------------------------- replicas (N > 1)
+def max_over_ranks(value: float, world: int, device) -> float:
+    """The slowest replica's figure: MAX all-reduce over the process group (identity for one rank).
+    `device`: where the reduction tensor lives ("cpu" with gloo, a CUDA device with NCCL)."""
+    if world <= 1:
+        return float(value)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_rate(world: int, P: int, nbytes: int, seconds_per_step: float) -> float:
+    """GB/s delivered by all replicas together: every replica delivers P*nbytes per step, and the
+    job is as slow as its slowest replica (`seconds_per_step` is already the max over ranks)."""
+    return world * P * nbytes / seconds_per_step / 1e9
+
+
 # --------------------------------------------------------------------------- the CUDA arm
 def run_ours(args):
     import numpy as np
@@ -209,10 +228,7 @@ def run_ours(args):
         total_ms = ev[0].elapsed_time(ev[steps])
         per = [ev[i].elapsed_time(ev[i + 1]) for i in range(steps)]
         clocks = sampler.stop(t_begin, t_end) if sampler else None
-        if world > 1:
-            t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            total_ms = float(t.item())
+        total_ms = max_over_ranks(total_ms, world, dev)
         return total_ms, per, clocks
 
     def check(plan_name):
@@ -233,7 +249,7 @@ def run_ours(args):
         launches = B.bcast_exec_num_launches(plan, mode)
         ms_step = total_ms / args.steps
         results[name] = dict(plan=plan, total_ms=total_ms, ms_step=ms_step, per=per, clocks=clocks, moved=moved,
-                             launches=launches, value=world * P * n / (ms_step * 1e-3) / 1e9)
+                             launches=launches, value=whole_job_rate(world, P, n, ms_step * 1e-3))
 
     tuned = results["tuned"]
     # roofline of the dominant kernel (WALK: the only kernel of a step)
@@ -268,14 +284,11 @@ def run_ours(args):
             B.bcast_exec_host(ptrs, plan, stream, mode, host_msg, outs)
         torch.cuda.synchronize()
         dt = time.perf_counter() - t0
-        if world > 1:
-            t = torch.tensor([dt], dtype=torch.float64, device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            dt = float(t.item())
+        dt = max_over_ranks(dt, world, dev)
         ok = bool((host_out[P - 1].numpy() == msg_np).all()) and bool((host_out[0].numpy() == msg_np).all())
         if not ok:
             raise SystemExit("e2e: host output differs from the message")
-        e2e = {"value": round(world * P * n / (dt / args.e2e_steps) / 1e9, 2), "unit": UNIT,
+        e2e = {"value": round(whole_job_rate(world, P, n, dt / args.e2e_steps), 2), "unit": UNIT,
                "h2d_bytes_per_step": n, "d2h_bytes_per_step": P * n, "steps": args.e2e_steps,
                "ms_per_step": round(dt / args.e2e_steps * 1e3, 3),
                "what": "bcast_exec_host: pinned host message -> root buffer, broadcast, all P rank buffers -> pinned host"}

@@ -48,23 +48,35 @@ def build(force: bool = False) -> str:
 _lib = None
 
 
+def _bind(path: str):
+    """Load a build of the oracle and declare its signatures."""
+    lib = ctypes.CDLL(path)
+    u64p = ctypes.POINTER(ctypes.c_uint64)
+    lib.oracle_bcast_simulate.restype = ctypes.c_int
+    lib.oracle_bcast_simulate.argtypes = [
+        ctypes.c_int, ctypes.c_int, ctypes.c_uint64, ctypes.c_int, ctypes.POINTER(ctypes.c_void_p),
+        ctypes.POINTER(ctypes.c_int64), ctypes.c_int64, ctypes.POINTER(ctypes.c_int64),
+        u64p, u64p, u64p, u64p]
+    lib.oracle_bcast_scatter_size.restype = ctypes.c_uint64
+    lib.oracle_bcast_scatter_size.argtypes = [ctypes.c_int, ctypes.c_uint64]
+    lib.oracle_bcast_step_flag.restype = ctypes.c_int
+    lib.oracle_bcast_step_flag.argtypes = [ctypes.c_int, ctypes.c_int,
+                                           ctypes.POINTER(ctypes.c_int), ctypes.POINTER(ctypes.c_int)]
+    return lib
+
+
 def _load():
     global _lib
     if _lib is None:
-        lib = ctypes.CDLL(build())
-        u64p = ctypes.POINTER(ctypes.c_uint64)
-        lib.oracle_bcast_simulate.restype = ctypes.c_int
-        lib.oracle_bcast_simulate.argtypes = [
-            ctypes.c_int, ctypes.c_int, ctypes.c_uint64, ctypes.c_int, ctypes.POINTER(ctypes.c_void_p),
-            ctypes.POINTER(ctypes.c_int64), ctypes.c_int64, ctypes.POINTER(ctypes.c_int64),
-            u64p, u64p, u64p, u64p]
-        lib.oracle_bcast_scatter_size.restype = ctypes.c_uint64
-        lib.oracle_bcast_scatter_size.argtypes = [ctypes.c_int, ctypes.c_uint64]
-        lib.oracle_bcast_step_flag.restype = ctypes.c_int
-        lib.oracle_bcast_step_flag.argtypes = [ctypes.c_int, ctypes.c_int,
-                                               ctypes.POINTER(ctypes.c_int), ctypes.POINTER(ctypes.c_int)]
-        _lib = lib
+        _lib = _bind(build())
     return _lib
+
+
+def use_build(path: str | None):
+    """Tests only: route all calls to another build of the oracle (a deliberately broken copy, to
+    show that the pins notice); ``None`` switches back to the real one."""
+    global _lib
+    _lib = _bind(path) if path else None
 
 
 class OracleError(RuntimeError):

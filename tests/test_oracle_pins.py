@@ -247,6 +247,23 @@ def test_broadcast_semantics(oracle, P, root, n, variant):
     assert ((ch >= 0) & (ch + nch <= P)).all()
 
 
+def test_schedule_geometry(oracle):
+    """Chunk c is bytes [min(cS, n), min((c+1)S, n)) with S = ceil(n / P) (Section IV listing); a
+    message carries whole chunks, never reaches past the message, and empty chunks still give
+    messages (of length 0, offset clipped to n)."""
+    for P, root, n, variant in [(8, 0, 4096, TUNED), (12, 5, 262144, NATIVE), (255, 254, 12288, TUNED),
+                                (10, 9, 7, NATIVE), (5, 2, 0, TUNED), (64, 17, (16 << 20) + 13, TUNED)]:
+        res = oracle.simulate(P, root, n, variant)
+        S = -(-n // P)
+        assert res.scatter_size == S
+        off, ln, ch, nch = res.col("offset"), res.col("len"), res.col("chunk"), res.col("nchunks")
+        assert ((off + ln) <= n).all() and (off >= 0).all() and (ln >= 0).all()
+        assert (off == np.minimum(ch * S, n)).all()
+        assert (off + ln == np.minimum((ch + nch) * S, n)).all()
+        assert ((ch >= 0) & (nch >= 1) & (ch + nch <= P)).all()
+        assert (res.msgs_recv.sum(axis=0)[[k for k in range(P) if k != root]] >= 1).all() or P == 1
+
+
 def test_validity_of_every_send(oracle):
     """A chunk is sent only after it has arrived at the sender: replay the schedule in order and
     check holdings; `dep` names the message that last delivered the chunk to the sender (-1: the
