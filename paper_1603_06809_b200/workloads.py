@@ -63,3 +63,27 @@ def message_bytes(seed: int, nbytes: int) -> np.ndarray:
 def poison_byte(rank: int) -> int:
     """Fill value for a non-root buffer before the broadcast; differs from rank to rank."""
     return (0x5A + 29 * rank) & 0xFF
+
+
+# ---- the paper's own experiment shapes (Section V), as a second workload set
+#: Experiment A: long messages, power-of-two process counts (Fig. 6)
+PAPER_A_P = (16, 64, 256)
+PAPER_A_NBYTES = (524288, 1 * MiB, 2 * MiB, 4 * MiB, 8 * MiB, 16 * MiB, 30_000_000)
+#: Experiment B: non-power-of-two process counts at the two MPICH thresholds and 1 MiB (Fig. 7)
+PAPER_B_P = (9, 17, 33, 65, 129)
+PAPER_B_NBYTES = (12288, 524287, 1048576)
+#: Experiment C: 129 processes, 12288 ... 2,560,000 bytes (Fig. 8)
+PAPER_C_P = 129
+PAPER_C_NBYTES = (12288, 65536, 262144, 524288, 1048576, 2_560_000)
+
+
+def paper_experiments() -> list[Workload]:
+    """Message sizes and process counts of the paper's three experiments; root 0 as in a plain
+    micro-benchmark.  Sizes between the end points that the paper names are a geometric fill."""
+    out = []
+    for P in PAPER_A_P:
+        out += [Workload(f"paperA_P{P}_{n}B", P, 0, n, BASE_SEED + 6) for n in PAPER_A_NBYTES]
+    for P in PAPER_B_P:
+        out += [Workload(f"paperB_P{P}_{n}B", P, 0, n, BASE_SEED + 7) for n in PAPER_B_NBYTES]
+    out += [Workload(f"paperC_P{PAPER_C_P}_{n}B", PAPER_C_P, 0, n, BASE_SEED + 8) for n in PAPER_C_NBYTES]
+    return out

@@ -154,6 +154,22 @@ def test_sweep_steps_executor_medium_points(oracle):
             check_against_oracle(oracle, wl, B.BCAST_TUNED, B.BCAST_EXEC_STEPS)
 
 
+# ---- the paper's own experiment shapes (Section V): every point element by element, both variants
+@pytest.mark.parametrize("variant", VARIANTS, ids=VARIANT_IDS)
+def test_paper_experiment_shapes(oracle, variant):
+    for wl in W.paper_experiments():
+        if wl.total_bytes <= 300 * W.MiB:
+            check_against_oracle(oracle, wl, variant, B.BCAST_EXEC_WALK)
+        else:
+            msg = W.message_bytes(wl.seed, wl.nbytes)
+            plan, bufs = run_broadcast(wl.P, wl.root, wl.nbytes, variant, B.BCAST_EXEC_WALK, msg)
+            assert bufs.all_equal_message() and bufs.guards_intact(), wl.name
+            ref = oracle.simulate(wl.P, wl.root, wl.nbytes, variant)
+            assert B.bcast_plan_total_bytes(plan) == int(ref.col("len").sum())
+            del bufs
+            torch.cuda.empty_cache()
+
+
 # ---- host-memory entry point
 @pytest.mark.parametrize("variant", VARIANTS, ids=VARIANT_IDS)
 def test_exec_host(oracle, variant):

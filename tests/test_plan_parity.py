@@ -89,6 +89,14 @@ def test_plan_equals_oracle_sweep(oracle, variant):
         assert_plan_equals_oracle(oracle, wl.P, wl.root, wl.nbytes, variant)
 
 
+@pytest.mark.parametrize("variant", [B.BCAST_NATIVE, B.BCAST_TUNED])
+def test_plan_equals_oracle_paper_experiment_shapes(oracle, variant):
+    shapes = W.paper_experiments()
+    assert len(shapes) == 3 * 7 + 5 * 3 + 6
+    for wl in shapes:
+        assert_plan_equals_oracle(oracle, wl.P, wl.root, wl.nbytes, variant)
+
+
 def test_plan_largest_rank_count(oracle):
     assert_plan_equals_oracle(oracle, B.BCAST_MAX_RANKS, 1000, 5_000_011, B.BCAST_TUNED)
 
