@@ -112,8 +112,9 @@ __device__ __forceinline__ Split split16(uint64_t lo, uint64_t hi)
 // The message is cut on a fixed grid of segments of 32 x U words (U x 512 bytes), and every
 // segment further at chunk boundaries: a slice is the part of one segment that lies in one chunk.
 // A warp owns a slice and walks it through the chunk's hop list on its own: warps never wait for
-// one another.  Slices are dealt round-robin (warp g takes slices g, g + G, ...), so neighbouring
-// warps work on neighbouring segments.  Lanes map to the fixed 16-byte words of the segment,
+// one another.  Slices are dealt round-robin with the block index running fastest (slice w goes to
+// block w mod G, then to that block's warp (w / G) mod 8): all SMs get the same share, and the
+// slices in flight at any time are neighbours in the message.  Lanes map to the fixed 16-byte words of the segment,
 // whatever the chunk's first byte is, so a warp's 512-byte accesses stay aligned to cache lines;
 // the <= 15 bytes before the first whole word and after the last one go one byte per lane.
 // The (src, dst) pair of hop h+1 is fetched while the loads of hop h are in flight.
@@ -129,7 +130,8 @@ bcast_walk_kernel(const __grid_constant__ RankPtrs<MAXP> bufs, const WalkSlice *
     const uint32_t lane = threadIdx.x & 31u;
     const long long total_warps = (long long)gridDim.x * kWarpsPerBlock;
 
-    for (long long w = (long long)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5); w < n_slices; w += total_warps) {
+    // slice w goes to block w mod gridDim.x: every SM gets the same number of slices (+-1)
+    for (long long w = (long long)(threadIdx.x >> 5) * gridDim.x + blockIdx.x; w < n_slices; w += total_warps) {
         const WalkSlice sl = slices[w];
         const uint64_t seg_lo = (uint64_t)sl.seg * kSeg, seg_hi = seg_lo + kSeg;
         const uint64_t lo = max(min((uint64_t)sl.chunk * scatter_size, nbytes), seg_lo);
@@ -429,17 +431,19 @@ int walk_blocks_per_sm(int u, int P, int *bps)
 }
 
 // Launch shape of the WALK executor: words per lane (U) and blocks.
-//   * Very few ranks (P <= 4): a slice makes at most three hops, the kernel is close to a plain
-//     copy and wants as many bytes in flight as the SMs can hold.
-//   * The whole message fits into the resident warps at once (one slice per warp): the run time is
-//     one walk down the longest hop list at memory latency, so take the smallest U that still fits
-//     -- the most warps, the fewest words each.
-//   * Otherwise the kernel is bound by the rate at which DRAM takes the scattered writes.  About
-//     32 KB in flight per SM (8 warps x 8 words x 512 B) saturate it; more concurrent slices only
-//     scatter the writes further.
-//     Every warp runs ceil(slices / warps) rounds; the fewest blocks that still need that many
-//     rounds are launched, so that all rounds are (almost) full instead of a last round that keeps
-//     a fraction of the GPU busy at memory latency.
+// Measured on B200: an SM's share of the work takes the same time whether 8 or 16 warps carry it
+// (the SM's load/store path is the limit), so what matters is that every SM gets the same share
+// -- the grid is a multiple of the SM count and slices are dealt SM by SM -- and that not more is
+// in flight than needed: about 32 KB per SM (8 warps x 8 words x 512 B) saturate the memory
+// system; more concurrent slices scatter the DRAM writes further and, with level-order hops,
+// push the copies that are still to be re-read out of L2.
+//   * Message larger than that (more than 1.4 rounds of SMs x 32 KB): U = 8, one block per SM,
+//     several rounds.
+//   * Smaller: everything is in flight at once and the run time is one walk down the longest hop
+//     list at memory latency; take the smallest U whose slices fit the resident warps (the most
+//     warps, the fewest words each).
+//   * Very few ranks (P <= 4): at most three hops per slice, close to a plain copy: as many
+//     bytes in flight as the SMs hold.
 // BCAST_WALK_WORDS and BCAST_WALK_BLOCKS_PER_SM override the choice (for experiments).
 struct WalkShape {
     int u = 1, grid = 1;
@@ -452,34 +456,32 @@ int choose_walk_shape(const bcast_plan_t &p, int sm_count, WalkShape *shape)
     const bool u_ok = forced_u == 1 || forced_u == 2 || forced_u == 4 || forced_u == 8;
     int rc, resident = 1, u = 0, bps = 0;
     if (u_ok || forced_bps > 0) {
-        u = u_ok ? forced_u : 4;
+        u = u_ok ? forced_u : 8;
         if ((rc = walk_blocks_per_sm(u, p.P, &resident))) return rc;
         bps = forced_bps > 0 ? std::min(forced_bps, resident) : resident;
     } else if (p.P <= 4) {
         u = 2;
         if ((rc = walk_blocks_per_sm(u, p.P, &resident))) return rc;
         bps = resident;
+    } else if (count_walk_slices(p, 8) * 5 > (long long)sm_count * kWarpsPerBlock * 7) {   // > 1.4 rounds
+        u = 8;
+        bps = 1;
     } else {
         for (int cand : {1, 2, 4, 8}) {
             if ((rc = walk_blocks_per_sm(cand, p.P, &resident))) return rc;
-            if (count_walk_slices(p, cand) <= (long long)sm_count * resident * kWarpsPerBlock) {
+            const long long slices = count_walk_slices(p, cand);
+            if (slices <= (long long)sm_count * resident * kWarpsPerBlock) {
                 u = cand;
-                bps = resident;
+                bps = (int)std::max<long long>(1, (slices + (long long)sm_count * kWarpsPerBlock - 1) /
+                                                      ((long long)sm_count * kWarpsPerBlock));
                 break;
             }
         }
-        if (!u) {
-            // eight words per lane; one block per SM once that alone gives six or more rounds
-            u = 8;
-            bps = count_walk_slices(p, u) >= 6ll * sm_count * kWarpsPerBlock ? 1 : 2;
-        }
+        if (!u) { u = 8; bps = 1; }
     }
     const long long slices = std::max<long long>(1, count_walk_slices(p, u));
-    const long long most = (long long)sm_count * std::max(1, bps) * kWarpsPerBlock;   // warps
-    const long long rounds = (slices + most - 1) / most;
-    const long long warps = (slices + rounds - 1) / rounds;
     shape->u = u;
-    shape->grid = (int)std::max<long long>(1, (warps + kWarpsPerBlock - 1) / kWarpsPerBlock);
+    shape->grid = (int)std::min<long long>(slices, (long long)sm_count * std::max(1, bps));
     return BCAST_OK;
 }
 
