@@ -55,11 +55,11 @@ def parse_args():
 # is reported as null until the counters are taken again.
 NCU_TRAFFIC = {
     # profiles/bcast_walk_kernel_P100_64MiB_launch_list_and_dram.md
-    ("cfg4", "walk"): {"dram_bytes_per_launch": 6.658e9,
-                       "exec_cu_sha256": "084fe303ec385a617f3d74dcdcd1ba494b6f1ac16bb06c1a8382149b4b7f48b0"},
+    ("cfg4", "walk"): {"dram_bytes_per_launch": 68208384 + 6586072832,
+                       "exec_cu_sha256": "7b45a1c16646bfd0bfccd1205492846dfb8035b46347f17b79ac1a99f40de454"},
     # profiles/bcast_walk_kernel_P64_16MiB_ncu_full.md
-    ("cfg3", "walk"): {"dram_bytes_per_launch": 1.018e9,
-                       "exec_cu_sha256": "084fe303ec385a617f3d74dcdcd1ba494b6f1ac16bb06c1a8382149b4b7f48b0"},
+    ("cfg3", "walk"): {"dram_bytes_per_launch": 17112064 + 1000195000,
+                       "exec_cu_sha256": "7b45a1c16646bfd0bfccd1205492846dfb8035b46347f17b79ac1a99f40de454"},
 }
 
 
