@@ -170,6 +170,64 @@ def test_paper_experiment_shapes(oracle, variant):
             torch.cuda.empty_cache()
 
 
+# ---- the largest accepted rank count (the P > 128 kernel instantiation with an 8 KiB pointer argument)
+@pytest.mark.parametrize("variant", VARIANTS, ids=VARIANT_IDS)
+def test_largest_rank_count(oracle, variant):
+    wl = W.Workload("P1024", B.BCAST_MAX_RANKS, 1000, 300_007, 77)
+    for mode in (B.BCAST_EXEC_WALK, B.BCAST_EXEC_WALK_PLAN_ORDER, B.BCAST_EXEC_STEPS):
+        check_against_oracle(oracle, wl, variant, mode)
+
+
+# ---- offsets beyond 4 GiB: 64-bit arithmetic in the planner, the slice list and the kernels
+def test_message_larger_than_4_gib(oracle):
+    P, root, n = 3, 2, (4 << 30) + 4097
+    msg = torch.empty(n, dtype=torch.uint8, device="cuda:0")
+    g = torch.Generator(device="cuda:0").manual_seed(5)
+    msg.random_(0, 256, generator=g)
+    bufs = [torch.full((n + 512,), 0xC3, dtype=torch.uint8, device="cuda:0") for _ in range(P)]
+    views = [b[256:256 + n] for b in bufs]
+    views[root].copy_(msg)
+    for mode in (B.BCAST_EXEC_WALK, B.BCAST_EXEC_STEPS):
+        for k in range(P):
+            if k != root:
+                views[k].fill_(W.poison_byte(k))
+        plan = B.bcast_plan(P, root, n, B.BCAST_TUNED)
+        B.bcast_exec_mode([v.data_ptr() for v in views], plan, torch.cuda.current_stream(), mode)
+        torch.cuda.synchronize()
+        for k in range(P):
+            assert torch.equal(views[k], msg)
+            assert bool((bufs[k][:256] == 0xC3).all()) and bool((bufs[k][256 + n:] == 0xC3).all())
+        ref = oracle.simulate(P, root, n, B.BCAST_TUNED)                 # schedule only
+        x = B.bcast_plan_xfers(plan)
+        assert np.array_equal(x["offset"].astype(np.int64), ref.col("offset"))
+        assert np.array_equal(x["len"].astype(np.int64), ref.col("len"))
+    del bufs, views, msg
+    torch.cuda.empty_cache()
+
+
+# ---- one plan, two sets of rank buffers, two streams at the same time
+def test_same_plan_on_two_streams_with_different_buffers(oracle):
+    wl = W.Workload("two_streams", 24, 7, 8 * W.MiB + 5, 91)
+    msg_a = W.message_bytes(wl.seed, wl.nbytes)
+    msg_b = W.message_bytes(wl.seed + 1, wl.nbytes)
+    a = RankBuffers(wl.P, wl.root, wl.nbytes, msg_a)
+    b = RankBuffers(wl.P, wl.root, wl.nbytes, msg_b)
+    plan = B.bcast_plan(wl.P, wl.root, wl.nbytes, B.BCAST_TUNED)
+    B.bcast_exec(a.pointers(), plan, torch.cuda.current_stream())     # first execution builds the tables
+    torch.cuda.synchronize()
+    a.reset()
+    torch.cuda.synchronize()
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    for _ in range(3):
+        B.bcast_exec(a.pointers(), plan, s1)
+        B.bcast_exec(b.pointers(), plan, s2)
+    torch.cuda.synchronize()
+    assert a.all_equal_message() and b.all_equal_message()
+    assert a.guards_intact() and b.guards_intact()
+    ref = oracle.simulate(wl.P, wl.root, wl.nbytes, B.BCAST_TUNED, message=msg_b)
+    assert np.array_equal(b.to_host(), ref.bufs)
+
+
 # ---- host-memory entry point
 @pytest.mark.parametrize("variant", VARIANTS, ids=VARIANT_IDS)
 def test_exec_host(oracle, variant):
@@ -190,6 +248,21 @@ def test_exec_host(oracle, variant):
         else:
             assert np.array_equal(got[k], ref.bufs[k])
     assert bufs.guards_intact()
+
+
+def test_exec_host_argument_errors():
+    wl = W.Workload("host_bad", 4, 1, 4096, 3)
+    bufs = RankBuffers(wl.P, wl.root, wl.nbytes, W.message_bytes(wl.seed, wl.nbytes))
+    plan = B.bcast_plan(wl.P, wl.root, wl.nbytes, B.BCAST_TUNED)
+    ptrs = (ctypes.c_void_p * 4)(*bufs.pointers())
+    st = ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+    assert B._lib.bcast_exec_host(ptrs, plan.handle, st, B.BCAST_EXEC_WALK, None, None) == B.BCAST_ERR_INVAL
+    assert B._lib.bcast_exec_host(None, plan.handle, st, B.BCAST_EXEC_WALK, None, None) == B.BCAST_ERR_INVAL
+    host = torch.from_numpy(W.message_bytes(9, wl.nbytes)).pin_memory()
+    assert B._lib.bcast_exec_host(ptrs, plan.handle, st, 99, ctypes.c_void_p(host.data_ptr()), None) == B.BCAST_ERR_INVAL
+    # an empty message needs no host pointer
+    empty = B.bcast_plan(4, 1, 0, B.BCAST_TUNED)
+    assert B._lib.bcast_exec_host(ptrs, empty.handle, st, B.BCAST_EXEC_WALK, None, None) == B.BCAST_OK
 
 
 # ---- argument errors are refused before anything is launched
