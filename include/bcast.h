@@ -42,8 +42,13 @@ extern "C" {
 
 #define BCAST_MAX_RANKS 1024 /* largest accepted P */
 
-enum { BCAST_NATIVE = 0, BCAST_TUNED = 1 };               /* variant: which ring allgather     */
-enum { BCAST_PHASE_SCATTER = 0, BCAST_PHASE_RING = 1 };   /* phase of a message                */
+/* variant: what follows the scatter.  NATIVE / TUNED: the ring allgather of Section III-A / IV.
+   DOUBLING: the recursive-doubling allgather that MPICH uses for medium messages on a power-of-two
+   number of processes (named in Section I; the standard hypercube exchange): log2 P exchanges, in
+   exchange i relative rank r swaps with r xor 2^i the block of 2^i chunks around each of them. */
+enum { BCAST_NATIVE = 0, BCAST_TUNED = 1, BCAST_DOUBLING = 2 };
+/* phase of a message; BCAST_PHASE_RING is the allgather phase (ring steps, or doubling exchanges) */
+enum { BCAST_PHASE_SCATTER = 0, BCAST_PHASE_RING = 1 };
 
 enum {
     BCAST_OK = 0,
@@ -78,12 +83,14 @@ enum {
 /* One message of the schedule.  Plain data, 48 bytes, host memory. */
 typedef struct {
     int32_t phase;     /* BCAST_PHASE_SCATTER or BCAST_PHASE_RING                                   */
-    int32_t step;      /* scatter: tree level 0..L-1 (L = ceil(log2 P)); ring: i-1 for ring step i   */
+    int32_t step;      /* scatter: tree level 0..L-1 (L = ceil(log2 P)); ring: i-1 for ring step i;
+                          doubling: exchange 0..log2(P)-1                                            */
     int32_t src_rank;  /* absolute rank whose buffer is read                                        */
     int32_t dst_rank;  /* absolute rank whose buffer is written                                     */
     int32_t chunk;     /* RELATIVE index of the (first) chunk carried; chunk c = bytes
                           [min(c*S, nbytes), min((c+1)*S, nbytes)) of the message                    */
-    int32_t nchunks;   /* ring: 1; scatter: the destination's own chunk plus its descendants'        */
+    int32_t nchunks;   /* ring: 1; scatter: the destination's own chunk plus its descendants';
+                          doubling exchange i: 2^i                                                   */
     uint64_t offset;   /* first byte, the same in the source and the destination buffer             */
     uint64_t len;      /* bytes; 0 for chunks past the end of a short message (still a message)      */
     int64_t dep;       /* index (into the plan's message array) of the message that last wrote this
@@ -102,7 +109,7 @@ typedef struct bcast_plan bcast_plan_t; /* opaque; created and freed by the libr
  *   P        number of ranks, 1..BCAST_MAX_RANKS.  P = 1 gives an empty plan.
  *   root     absolute rank that owns the message, 0..P-1
  *   nbytes   message size; 0 is valid (all messages have len 0)
- *   variant  BCAST_NATIVE or BCAST_TUNED
+ *   variant  BCAST_NATIVE, BCAST_TUNED, or BCAST_DOUBLING (P must then be a power of two)
  *   out      host pointer that receives the plan; the caller releases it with bcast_plan_free()
  * Messages are ordered by (phase, step, dst_rank); a rank receives at most one message per step.
  * Errors: BCAST_ERR_INVAL (arguments out of range, out == NULL), BCAST_ERR_NOMEM.
@@ -121,7 +128,7 @@ int32_t bcast_plan_variant(const bcast_plan_t *plan);
 uint64_t bcast_plan_nbytes(const bcast_plan_t *plan);
 uint64_t bcast_plan_scatter_size(const bcast_plan_t *plan);      /* S = ceil(nbytes / P) (Section IV listing) */
 int64_t bcast_plan_num_xfers(const bcast_plan_t *plan);          /* number of messages               */
-int32_t bcast_plan_num_steps(const bcast_plan_t *plan);          /* L + (P-1); 0 for P = 1           */
+int32_t bcast_plan_num_steps(const bcast_plan_t *plan);          /* L + (P-1) (doubling: 2L); 0 for P = 1 */
 const bcast_xfer_t *bcast_plan_xfers(const bcast_plan_t *plan);  /* [num_xfers], canonical order      */
 const int64_t *bcast_plan_step_begin(const bcast_plan_t *plan);  /* [num_steps+1]: messages of step s
                                                                     are [step_begin[s], step_begin[s+1]) */

@@ -17,6 +17,14 @@
  *   - Section IV (Figs. 4-5 and the pseudo-code listing): tuned "non-enclosed"
  *     ring allgather; each process computes (step, flag) and turns send-only or
  *     receive-only once  step > P - i.
+ *   - Section I: for medium messages on a power-of-two number of processes MPICH
+ *     follows the scatter with a recursive-doubling allgather instead of the ring.
+ *     The paper only names it; the exchange pattern simulated here is the standard
+ *     one of that algorithm (Thakur, Rabenseifner, Gropp, "Optimization of
+ *     Collective Communication Operations in MPICH"): in step i = 0..log2(P)-1 a
+ *     process exchanges, with the process whose relative rank differs in bit i, the
+ *     block of 2^i chunks that starts at its own relative rank with the low i bits
+ *     cleared.  Third variant (2); power-of-two P only.
  *
  * Every simulated process runs the per-process logic of the listing; a message
  * is the pair of one process's send and its right neighbour's receive, and the
@@ -41,7 +49,10 @@
  *
  * Pinned by tests/test_oracle_pins.py against the worked examples of
  * Figs. 1-5, the printed message counts, closed forms, MPI broadcast
- * semantics and a brute-force ownership enumeration.  Nothing is unpinned.
+ * semantics and a brute-force ownership enumeration; the recursive-doubling
+ * variant, for which the paper prints nothing, against the textbook hypercube
+ * exchange with explicit ownership sets, its byte budget, and the two-process
+ * case where it must coincide with the ring.  Nothing is unpinned.
  */
 #include <stdint.h>
 #include <stdlib.h>
@@ -239,10 +250,43 @@ out:
     return rc;
 }
 
+/* Section I (named only) -- recursive-doubling allgather after the scatter; P a power of two. */
+static int doubling_phase(sim_t *s, pending_t *m)
+{
+    const int P = s->P;
+    int rc = ORC_OK;
+    int *wants_from = malloc(sizeof(int) * (size_t)P), *wants_chunk = malloc(sizeof(int) * (size_t)P);
+    if (!wants_from || !wants_chunk) { rc = ORC_E_NOMEM; goto out; }
+    for (int i = 0, mask = 1; mask < P; i++, mask <<= 1) {
+        /* every process posts its receive: from the partner, the partner's current block */
+        for (int k = 0; k < P; k++) {
+            const int r = rel_of(s, k), partner = r ^ mask;
+            wants_from[k] = abs_of(s, partner);
+            wants_chunk[k] = (partner >> i) << i;
+        }
+        /* every process sends its own current block to the partner */
+        int nm = 0;
+        for (int k = 0; k < P; k++) {
+            const int r = rel_of(s, k), partner = abs_of(s, r ^ mask);
+            const int my_block = (r >> i) << i;
+            if (wants_from[partner] != k || wants_chunk[partner] != my_block) { rc = ORC_E_UNMATCHED; goto out; }
+            m[nm].src = k; m[nm].dst = partner; m[nm].chunk = my_block; m[nm].nchunks = mask;
+            nm++;
+        }
+        rc = deliver_step(s, PH_RING, i, m, nm);
+        if (rc) goto out;
+    }
+out:
+    free(wants_from); free(wants_chunk);
+    return rc;
+}
+
 /*
  * Simulate one broadcast.
  *   P, root, nbytes   communicator size, root rank, message bytes
- *   tuned             0: native ring (Section III-A), 1: tuned ring (Section IV)
+ *   tuned             0: native ring (Section III-A), 1: tuned ring (Section IV),
+ *                     2: recursive-doubling allgather in place of the ring (Section I; P must be
+ *                        a power of two)
  *   buf               P host buffers of nbytes each; buf[root] holds the message.  NULL: no data is
  *                     moved, only the schedule and the counters are produced.
  *   sched, cap        room for cap records of 9 int64 (phase, step, src, dst, chunk, nchunks,
@@ -258,6 +302,7 @@ int oracle_bcast_simulate(int P, int root, uint64_t nbytes, int tuned, uint8_t *
     if (P < 1 || root < 0 || root >= P || !sched || !nsched || cap < 0 ||
         !bytes_sent || !bytes_recv || !msgs_sent || !msgs_recv)
         return ORC_E_ARG;
+    if (tuned < 0 || tuned > 2 || (tuned == 2 && (P & (P - 1)) != 0)) return ORC_E_ARG;
 
     sim_t s;
     memset(&s, 0, sizeof s);
@@ -285,7 +330,7 @@ int oracle_bcast_simulate(int P, int root, uint64_t nbytes, int tuned, uint8_t *
 
     rc = scatter_phase(&s, L, m);
     if (rc) goto out;
-    rc = ring_phase(&s, tuned, m);
+    rc = tuned == 2 ? doubling_phase(&s, m) : ring_phase(&s, tuned, m);
     if (rc) goto out;
 
     /* MPI broadcast semantics (Section III-A): on return every process has the root's message */

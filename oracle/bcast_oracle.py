@@ -20,7 +20,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "bcast_oracle.c")
 _LIB = os.path.join(_HERE, "_build", "libbcast_oracle.so")
 
-NATIVE, TUNED = 0, 1
+NATIVE, TUNED, DOUBLING = 0, 1, 2
 SCATTER, RING = 0, 1
 SEND_ONLY, RECV_ONLY = 0, 1
 

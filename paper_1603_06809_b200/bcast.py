@@ -19,7 +19,7 @@ if not os.path.exists(_LIB_PATH):
 _lib = ctypes.CDLL(_LIB_PATH)
 
 BCAST_MAX_RANKS = 1024
-BCAST_NATIVE, BCAST_TUNED = 0, 1
+BCAST_NATIVE, BCAST_TUNED, BCAST_DOUBLING = 0, 1, 2
 BCAST_PHASE_SCATTER, BCAST_PHASE_RING = 0, 1
 BCAST_OK, BCAST_ERR_INVAL, BCAST_ERR_NOMEM, BCAST_ERR_CUDA, BCAST_ERR_CAPACITY = 0, -1, -2, -3, -4
 BCAST_STATIC_SCRATCH_BYTES = 2 << 20

@@ -7,6 +7,9 @@
 // scatter (Section III-A, Figs. 1-2), and in ring step i receives chunk (r - i) mod P from its
 // left neighbour (Section III-A, Fig. 3).  The tuned ring (Section IV) keeps exactly the receives
 // of chunks outside [r, r + s(r)), i.e. steps i <= P - s(r); the root (s = P) never receives.
+// The recursive-doubling variant (Section I; power-of-two P) replaces the ring by log2 P exchanges:
+// in exchange i relative rank r receives from r xor 2^i the block of 2^i chunks that starts at the
+// partner's rank with its low i bits cleared.
 #include <algorithm>
 #include <new>
 
@@ -44,11 +47,12 @@ void build(bcast_plan_t &p)
     }
     p.L = 0;
     while ((1 << p.L) < P) p.L++;
-    const int nsteps = P > 1 ? p.L + (P - 1) : 0;
+    const bool doubling = p.variant == BCAST_DOUBLING;
+    const int nsteps = P > 1 ? p.L + (doubling ? p.L : P - 1) : 0;
     p.step_begin.assign(nsteps + 1, 0);
     if (P == 1) return;
 
-    size_t ring_msgs = (size_t)P * (P - 1);
+    size_t ring_msgs = doubling ? (size_t)P * p.L : (size_t)P * (P - 1);
     if (p.variant == BCAST_TUNED) {
         ring_msgs = (size_t)P * P;
         for (int r = 0; r < P; r++) ring_msgs -= g.subtree(r);
@@ -80,6 +84,43 @@ void build(bcast_plan_t &p)
             count(p, x);
             p.xfers.push_back(x);
         }
+    }
+
+    if (doubling) {
+        // ---- recursive doubling: exchange i, receiver r takes the block of 2^i chunks from r xor 2^i
+        std::vector<std::vector<int64_t>> into(p.L, std::vector<int64_t>(P, -1));   // [exchange][relative rank]
+        for (int i = 0; i < p.L; i++) {
+            const int mask = 1 << i;
+            p.step_begin[p.L + i] = (int64_t)p.xfers.size();
+            for (int k = 0; k < P; k++) {
+                const int r = g.rel_rank(k), q = r ^ mask;     // receiver, sender (relative)
+                const int block = (q >> i) << i;
+                bcast_xfer_t x{};
+                x.phase = BCAST_PHASE_RING;
+                x.step = i;
+                x.src_rank = g.abs_rank(q);
+                x.dst_rank = k;
+                x.chunk = block;
+                x.nchunks = mask;
+                x.offset = g.chunk_begin(block);
+                x.len = g.chunk_begin(block + mask) - x.offset;
+                // who last wrote the block's first chunk into the sender: the exchange that brought it
+                // the sub-block starting there (the highest set bit of q below bit i), else the scatter
+                const int low = q & (mask - 1);
+                if (low == 0) {
+                    x.dep = delivered[q];
+                } else {
+                    int j = 0;
+                    while ((2 << j) <= low) j++;
+                    x.dep = into[j][q];
+                }
+                into[i][r] = (int64_t)p.xfers.size();
+                count(p, x);
+                p.xfers.push_back(x);
+            }
+        }
+        p.step_begin[nsteps] = (int64_t)p.xfers.size();
+        return;
     }
 
     // ---- ring: step i, receiver r takes chunk (r - i) mod P from r - 1
@@ -122,7 +163,8 @@ int bcast_plan(int P, int root, uint64_t nbytes, int variant, bcast_plan_t **out
     if (!out) return BCAST_ERR_INVAL;
     *out = nullptr;
     if (P < 1 || P > BCAST_MAX_RANKS || root < 0 || root >= P) return BCAST_ERR_INVAL;
-    if (variant != BCAST_NATIVE && variant != BCAST_TUNED) return BCAST_ERR_INVAL;
+    if (variant != BCAST_NATIVE && variant != BCAST_TUNED && variant != BCAST_DOUBLING) return BCAST_ERR_INVAL;
+    if (variant == BCAST_DOUBLING && (P & (P - 1)) != 0) return BCAST_ERR_INVAL;
     if (nbytes > (UINT64_MAX >> 1) - (uint64_t)P) return BCAST_ERR_INVAL;
     bcast_plan_t *p = nullptr;
     try {

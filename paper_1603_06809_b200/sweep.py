@@ -3,7 +3,8 @@
     python -m paper_1603_06809_b200.sweep [--set config5|paper|configs] [--mode walk|walk_plan_order|steps|graph]
                                            [--iters N] [--json]
 
-For every workload: median time of the tuned and of the native variant (CUDA events around each
+For every workload: median time of the tuned and of the native variant (and, where P is a power of
+two, of the scatter + recursive-doubling variant) (CUDA events around each
 execution, after warm-up), the effective broadcast rate P*nbytes/t, the algorithmic rate
 2*sum(len)/t, and the tuned-over-native speed-up.  After timing, every rank buffer is compared with
 the root's message on the device.  Uses only the CUDA library: no CPU path is involved.
@@ -55,8 +56,12 @@ def run(workloads, mode: int, iters: int):
         it = iters if wl.total_bytes < (1 << 30) else max(5, iters // 5)
         t_ms, t_bytes = time_workload(wl, B.BCAST_TUNED, mode, it)
         n_ms, n_bytes = time_workload(wl, B.BCAST_NATIVE, mode, it)
+        d_ms = None
+        if wl.P & (wl.P - 1) == 0:                       # recursive doubling needs a power of two
+            d_ms, _ = time_workload(wl, B.BCAST_DOUBLING, mode, it)
         rows.append({
             "workload": wl.name, "P": wl.P, "nbytes": wl.nbytes,
+            "doubling_us": None if d_ms is None else round(d_ms * 1e3, 2),
             "tuned_us": round(t_ms * 1e3, 2), "native_us": round(n_ms * 1e3, 2),
             "tuned_effective_GBps": round(wl.P * wl.nbytes / t_ms / 1e6, 1),
             "tuned_algorithmic_GBps": round(2 * t_bytes / t_ms / 1e6, 1),
@@ -85,10 +90,11 @@ def main():
             print(json.dumps(r))
         return
     print(f"{'workload':28s} {'tuned us':>10s} {'native us':>10s} {'P*n/t GB/s':>11s} {'alg GB/s':>10s} "
-          f"{'bytes n/t':>9s} {'speed-up':>8s}")
+          f"{'bytes n/t':>9s} {'speed-up':>8s} {'doubling us':>11s}")
     for r in rows:
         print(f"{r['workload']:28s} {r['tuned_us']:10.2f} {r['native_us']:10.2f} {r['tuned_effective_GBps']:11.1f} "
-              f"{r['tuned_algorithmic_GBps']:10.1f} {r['bytes_native_over_tuned']:9.4f} {r['speedup_tuned_over_native']:8.4f}")
+              f"{r['tuned_algorithmic_GBps']:10.1f} {r['bytes_native_over_tuned']:9.4f} {r['speedup_tuned_over_native']:8.4f} "
+              f"{'' if r['doubling_us'] is None else format(r['doubling_us'], '11.2f')}")
 
 
 if __name__ == "__main__":

@@ -170,6 +170,18 @@ def test_paper_experiment_shapes(oracle, variant):
             torch.cuda.empty_cache()
 
 
+# ---- scatter + recursive-doubling allgather (power-of-two P), every executor
+DOUBLING_CASES = [W.CFG1, W.CFG3, W.Workload("P2", 2, 1, 4097, 21), W.Workload("P4", 4, 3, 3, 22),
+                  W.Workload("P16_odd", 16, 5, 1_000_003, 23), W.Workload("P32", 32, 0, 12288, 24),
+                  W.Workload("P256", 256, 255, 4 * W.MiB + 1, 25), W.Workload("P128_empty", 128, 9, 100, 26)]
+
+
+@pytest.mark.parametrize("mode", MODES, ids=MODE_IDS)
+@pytest.mark.parametrize("wl", DOUBLING_CASES, ids=lambda w: w.name)
+def test_recursive_doubling_variant(oracle, wl, mode):
+    check_against_oracle(oracle, wl, B.BCAST_DOUBLING, mode)
+
+
 # ---- the largest accepted rank count (the P > 128 kernel instantiation with an 8 KiB pointer argument)
 @pytest.mark.parametrize("variant", VARIANTS, ids=VARIANT_IDS)
 def test_largest_rank_count(oracle, variant):

@@ -31,6 +31,9 @@ MUTANTS = [
      "s->bytes_sent[(size_t)phase * P + m[a].dst] += len;"),
     ("empty_messages_dropped_from_counts", "s->msgs_recv[(size_t)phase * P + m[a].dst] += 1;",
      "s->msgs_recv[(size_t)phase * P + m[a].dst] += len ? 1 : 0;"),
+    ("doubling_sends_one_chunk_of_the_block", "m[nm].nchunks = mask;", "m[nm].nchunks = 1;"),
+    ("doubling_partner_by_relative_rank", "wants_from[k] = abs_of(s, partner);", "wants_from[k] = partner;"),
+    ("doubling_block_of_the_wrong_size", "const int my_block = (r >> i) << i;", "const int my_block = (r >> (i + 1)) << (i + 1);"),
     ("offset_not_clipped", "static uint64_t chunk_begin(const sim_t *s, int c) { return umin((uint64_t)c * s->S, s->n); }",
      "static uint64_t chunk_begin(const sim_t *s, int c) { return (uint64_t)c * s->S; }"),
 ]
@@ -55,6 +58,12 @@ def schedule_level_pins(oracle):
     yield lambda: pins.test_tuned_is_subset_of_native(oracle)
     yield lambda: pins.test_root_rotation(oracle)
     yield lambda: pins.test_schedule_geometry(oracle)
+    yield lambda: pins.test_doubling_equals_ring_for_two_processes(oracle)
+    for P in (1, 2, 8, 64):
+        yield lambda P=P: pins.test_doubling_against_textbook_hypercube_exchange(oracle, P)
+    for case in ((4, 1, 3), (16, 15, 65521), (64, 17, (16 << 20) + 13)):
+        yield lambda case=case: pins.test_doubling_byte_budget_and_semantics(oracle, *case, with_data=False)
+    yield lambda: pins.test_doubling_root_rotation_and_validity(oracle)
 
 
 def test_the_unbroken_oracle_passes_the_same_pins(oracle):

@@ -344,3 +344,95 @@ def test_degenerate_inputs(oracle):
         oracle.simulate(4, 4, 10, TUNED)
     with pytest.raises(oracle.OracleError):
         oracle.simulate(0, 0, 10, TUNED)
+
+
+# ----------------------------------------------------------------------------- recursive doubling
+DOUBLING = 2
+
+
+def test_doubling_equals_ring_for_two_processes(oracle):
+    """With two processes the one exchange of recursive doubling is the one step of the ring (each
+    sends its own chunk to the other): the schedules must be identical, `dep` included."""
+    for root, n in ((0, 10), (1, 10), (1, 1), (0, 4097)):
+        a = oracle.simulate(2, root, n, NATIVE)
+        b = oracle.simulate(2, root, n, DOUBLING)
+        assert np.array_equal(a.schedule, b.schedule)
+        assert np.array_equal(a.bytes_recv, b.bytes_recv) and np.array_equal(a.msgs_sent, b.msgs_sent)
+
+
+@pytest.mark.parametrize("P", [1, 2, 4, 8, 16, 32, 64, 256])
+def test_doubling_against_textbook_hypercube_exchange(oracle, P):
+    """Section I names the recursive-doubling allgather; its textbook definition: in step i every
+    process exchanges with the process whose (relative) rank differs in bit i everything both have
+    gathered so far, i.e. the aligned block of 2^i chunks around each of them, so that after step i
+    every process holds the aligned block of 2^(i+1) chunks around itself.  Checked with explicit
+    ownership sets on top of the scatter's holdings."""
+    root, n = P // 3, 11 * P + 5
+    res = oracle.simulate(P, root, n, DOUBLING)
+    lg = P.bit_length() - 1
+    rows = rel_rows(res, RING)
+    assert len(rows) == P * lg
+    holds = [set(range(r, r + subtree(P, r))) for r in range(P)]
+    for i in range(lg):
+        step = [m for m in rows if m[0] == i + 1]
+        assert len(step) == P
+        assert sorted(m[2] for m in step) == list(range(P))        # everybody receives once
+        arriving = {}
+        for _, src, dst, c, nc in step:
+            assert dst == src ^ (1 << i)                           # partner differs in bit i
+            block = set(range(c, c + nc))
+            assert block == set(range((src >> i) << i, ((src >> i) << i) + (1 << i)))
+            assert block <= holds[src]                             # the sender has gathered it
+            arriving[dst] = block
+        for r in range(P):
+            holds[r] |= arriving[r]
+            lo = (r >> (i + 1)) << (i + 1)
+            assert set(range(lo, lo + (2 << i))) <= holds[r]
+    assert all(h == set(range(P)) for h in holds)
+
+
+@pytest.mark.parametrize("P,root,n", [(4, 1, 3), (8, 0, 1 << 20), (16, 15, 65521), (64, 17, (16 << 20) + 13), (256, 255, 12288)])
+def test_doubling_byte_budget_and_semantics(oracle, P, root, n, with_data=True):
+    """Every process receives, over the log2 P exchanges, each chunk but its own exactly once: n minus
+    its own chunk's bytes, (P-1)*n in total for the phase -- as many bytes as the native ring moves,
+    in log2 P steps instead of P-1.  With data: every buffer ends up equal to the root's message."""
+    small = with_data and n <= (1 << 20)
+    msg = np.random.default_rng(P).integers(0, 256, size=n, dtype=np.uint8) if small else None
+    res = oracle.simulate(P, root, n, DOUBLING, message=msg)
+    S = -(-n // P)
+
+    def span(a, b):
+        return min(b * S, n) - min(a * S, n)
+    assert int(res.col("len")[res.col("phase") == RING].sum()) == (P - 1) * n
+    for k in range(P):
+        r = (k - root) % P
+        assert int(res.bytes_recv[RING, k]) == n - span(r, r + 1)
+        assert int(res.bytes_sent[RING, k]) == sum(span((r >> i) << i, ((r >> i) << i) + (1 << i)) for i in range(P.bit_length() - 1))
+        assert int(res.msgs_recv[RING, k]) == int(res.msgs_sent[RING, k]) == P.bit_length() - 1
+    nat = oracle.simulate(P, root, n, NATIVE)
+    assert np.array_equal(res.phase_rows(SCATTER), nat.phase_rows(SCATTER))      # same scatter
+    if small:
+        assert (res.bufs == msg[None, :]).all()
+
+
+def test_doubling_needs_power_of_two(oracle):
+    for P in (3, 6, 12, 100, 255):
+        with pytest.raises(oracle.OracleError):
+            oracle.simulate(P, 0, 1000, DOUBLING)
+    with pytest.raises(oracle.OracleError):
+        oracle.simulate(8, 0, 1000, 3)
+
+
+def test_doubling_root_rotation_and_validity(oracle):
+    P, n = 16, 12345
+    base = oracle.simulate(P, 0, n, DOUBLING)
+    base_rows = sorted(tuple(int(v) for v in r[:8]) for r in base.schedule)
+    for root in range(P):
+        res = oracle.simulate(P, root, n, DOUBLING)
+        rows = sorted((int(r[0]), int(r[1]), (int(r[2]) - root) % P, (int(r[3]) - root) % P,
+                       int(r[4]), int(r[5]), int(r[6]), int(r[7])) for r in res.schedule)
+        assert rows == base_rows
+        keys = [(int(r[0]), int(r[1]), int(r[3])) for r in res.schedule]
+        assert keys == sorted(keys) and len(set(keys)) == len(keys)
+        for x, row in enumerate(res.schedule):
+            assert -1 <= int(row[8]) < x

@@ -37,7 +37,7 @@ def assert_plan_equals_oracle(oracle, P, root, n, variant):
     # CSR over steps: L + P - 1 steps, each holding the messages with that (phase, step)
     sb = B.bcast_plan_step_begin(plan)
     L = (P - 1).bit_length()
-    nsteps = L + P - 1 if P > 1 else 0
+    nsteps = (2 * L if variant == B.BCAST_DOUBLING else L + P - 1) if P > 1 else 0
     assert B.bcast_plan_num_steps(plan) == nsteps and len(sb) == nsteps + 1
     assert sb[0] == 0 and sb[-1] == len(mine) and (np.diff(sb) >= 0).all()
     for s in range(nsteps):
@@ -97,13 +97,27 @@ def test_plan_equals_oracle_paper_experiment_shapes(oracle, variant):
         assert_plan_equals_oracle(oracle, wl.P, wl.root, wl.nbytes, variant)
 
 
+def test_plan_equals_oracle_doubling(oracle):
+    """Scatter + recursive-doubling allgather (power-of-two P): schedule, `dep` and counters."""
+    for P in (1, 2, 4, 8, 16, 32, 64, 128, 256, 1024):
+        for root in sorted({0, P // 3, P - 1}):
+            for n in (0, 1, P - 1, P, P + 1, 12288, 1000003):
+                assert_plan_equals_oracle(oracle, P, root, n, B.BCAST_DOUBLING)
+    for wl in (W.CFG1, W.CFG3):
+        assert_plan_equals_oracle(oracle, wl.P, wl.root, wl.nbytes, B.BCAST_DOUBLING)
+    for P in (3, 12, 100, 255):
+        with pytest.raises(B.BcastError) as e:
+            B.bcast_plan(P, 0, 1000, B.BCAST_DOUBLING)
+        assert e.value.code == B.BCAST_ERR_INVAL
+
+
 def test_plan_largest_rank_count(oracle):
     assert_plan_equals_oracle(oracle, B.BCAST_MAX_RANKS, 1000, 5_000_011, B.BCAST_TUNED)
 
 
 def test_plan_argument_errors():
     for args in [(0, 0, 10, 1), (-1, 0, 10, 1), (B.BCAST_MAX_RANKS + 1, 0, 10, 1), (4, 4, 10, 1), (4, -1, 10, 1),
-                 (4, 0, 10, 2), (4, 0, 10, -1), (4, 0, 2**64 - 1, 1)]:
+                 (4, 0, 10, 3), (4, 0, 10, -1), (4, 0, 2**64 - 1, 1)]:
         with pytest.raises(B.BcastError) as e:
             B.bcast_plan(*args)
         assert e.value.code == B.BCAST_ERR_INVAL
@@ -142,7 +156,7 @@ def test_exec_without_gpu_fails_loudly():
     assert e.value.code == B.BCAST_ERR_CUDA
 
 
-@pytest.mark.parametrize("variant", [B.BCAST_NATIVE, B.BCAST_TUNED])
+@pytest.mark.parametrize("variant", [B.BCAST_NATIVE, B.BCAST_TUNED, B.BCAST_DOUBLING])
 def test_walk_order_respects_every_dependency(oracle, variant):
     """The order in which the one-launch executor performs the messages of a chunk (both of its
     modes): the same messages as the oracle's schedule has for that chunk, each once; a message
@@ -150,6 +164,8 @@ def test_walk_order_respects_every_dependency(oracle, variant):
     the chunk already and in the end every rank holds it."""
     for P, root, n in [(2, 1, 64), (8, 0, 1 << 12), (10, 3, 12345), (12, 5, 256 << 10), (33, 32, 100003),
                        (64, 17, (16 << 20) + 13), (100, 63, 64 << 20), (255, 254, 12288)]:
+        if variant == B.BCAST_DOUBLING and P & (P - 1):
+            continue
         plan = B.bcast_plan(P, root, n, variant)
         ref = oracle.simulate(P, root, n, variant)
         S = ref.scatter_size
@@ -169,8 +185,10 @@ def test_walk_order_respects_every_dependency(oracle, variant):
                 holders = {root}
                 for m in order:
                     dep = int(sched[m, 8])
-                    if dep >= 0:
-                        assert dep in pos and pos[dep] < pos[int(m)]
+                    if variant != B.BCAST_DOUBLING:
+                        assert dep < 0 or dep in pos       # the producer covers this chunk too
+                    if dep in pos:                         # (doubling: `dep` is about the block's first chunk)
+                        assert pos[dep] < pos[int(m)]
                     assert int(sched[m, 2]) in holders
                     holders.add(int(sched[m, 3]))
                 if want:
