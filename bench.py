@@ -55,11 +55,11 @@ def parse_args():
 # is reported as null until the counters are taken again.
 NCU_TRAFFIC = {
     # profiles/bcast_walk_kernel_P100_64MiB_launch_list_and_dram.md
-    ("cfg4", "walk"): {"dram_bytes_per_launch": 68208384 + 6586072832,
-                       "exec_cu_sha256": "7b45a1c16646bfd0bfccd1205492846dfb8035b46347f17b79ac1a99f40de454"},
-    # profiles/bcast_walk_kernel_P64_16MiB_ncu_full.md
-    ("cfg3", "walk"): {"dram_bytes_per_launch": 17112064 + 1000195000,
-                       "exec_cu_sha256": "7b45a1c16646bfd0bfccd1205492846dfb8035b46347f17b79ac1a99f40de454"},
+    ("cfg4", "walk"): {"dram_bytes_per_launch": 68298752 + 6586297856,
+                       "exec_cu_sha256": "2b99f7d17361560fd69fbb595060452d5fa3e6d68febc40b046cd653b3041b40"},
+    # profiles/bcast_walk_kernel_P64_16MiB_ncu_full.md (same one-pass metric pair, cfg3)
+    ("cfg3", "walk"): {"dram_bytes_per_launch": 17127424 + 998557952,
+                       "exec_cu_sha256": "2b99f7d17361560fd69fbb595060452d5fa3e6d68febc40b046cd653b3041b40"},
 }
 
 

@@ -9,13 +9,14 @@
 //   * a byte of the message at some rank depends only on the same byte at the rank it is copied
 //     from, so messages that cover different byte ranges never depend on one another.
 //
-// WALK executor (one launch): the message is cut into tiles on a fixed grid of byte offsets, split
-// further at chunk boundaries.  A warp takes a slice of a tile and performs, in plan order, every
-// message that covers the tile's chunk, restricted to the slice: load from the source rank's
-// buffer, store to the destination rank's buffer.  Each thread always handles the same bytes of
-// the slice, so the load of hop h+1 reads what the same thread stored in hop h or earlier:
-// program order per thread is the only ordering the schedule needs.  Loads bypass L1 (.cg) so that
-// every hop really re-reads the source rank's buffer from the L2/HBM level.
+// WALK executor (one launch): the message is cut into segments on a fixed grid of byte offsets,
+// split further at chunk boundaries.  A warp takes such a slice and performs every message of the
+// plan that covers the slice's chunk, restricted to the slice, in an order that respects the
+// plan's dependencies: load from the source rank's buffer, store to the destination rank's
+// buffer.  Each thread always handles the same bytes of the slice, so whatever a hop reads was
+// stored earlier by the same thread: program order per thread is the only ordering the schedule
+// needs.  Loads bypass L1 (.cg) so that every hop really re-reads the source rank's buffer from
+// the L2/HBM level.
 //
 // STEPS / GRAPH executors: one launch per plan step, the messages of the step cut into tiles.
 #include <cuda_runtime.h>
@@ -241,7 +242,6 @@ struct bcast_device_state {
     // STEPS / GRAPH
     DevXfer *d_xfers = nullptr;
     std::vector<StepLaunch> steps;
-    int64_t nonempty_steps = 0;
     cudaGraph_t graph = nullptr;
     cudaGraphExec_t graph_exec = nullptr;
     std::vector<void *> graph_bufs;
@@ -307,7 +307,6 @@ int build_step_tables(const bcast_plan_t &p, bcast_device_state &ds)
     }
     const int nsteps = (int)p.step_begin.size() - 1;
     ds.steps.resize(nsteps);
-    ds.nonempty_steps = 0;
     for (int s = 0; s < nsteps; s++) {
         StepLaunch sl{p.step_begin[s], (unsigned)(p.step_begin[s + 1] - p.step_begin[s]), 0u};
         for (int64_t i = p.step_begin[s]; i < p.step_begin[s + 1]; i++) {
@@ -317,7 +316,6 @@ int build_step_tables(const bcast_plan_t &p, bcast_device_state &ds)
             sl.tiles = std::max<unsigned>(sl.tiles, (unsigned)t);
         }
         ds.steps[s] = sl;
-        ds.nonempty_steps += sl.tiles > 0;
     }
     return upload(&ds.d_xfers, hx);
 }
