@@ -60,8 +60,9 @@ enum {
 
 /* How bcast_exec_mode() runs a plan.  All modes perform exactly the plan's messages. */
 enum {
-    /* One launch for the whole plan.  The message is cut into tiles on a fixed grid of byte
-       offsets; a warp takes a slice of a tile and carries it through every message of the plan
+    /* One launch for the whole plan.  The message is cut into segments on a fixed grid of byte
+       offsets (and at chunk boundaries); a warp takes such a slice and carries it through every
+       message of the plan
        that covers it (scatter hops and ring hops), re-reading it from the source rank's buffer at
        every hop.  Messages that cover different byte ranges are independent, so no waiting
        between warps is needed.  The hops of a slice run in an order that respects every `dep`
@@ -189,14 +190,15 @@ int bcast_exec_host(void *const *rank_bufs, const bcast_plan_t *plan, void *cuda
  * services that run under a fixed memory budget, and latency-critical code for which the implicit
  * device-wide synchronisation of cudaMalloc / cudaFree is not acceptable.  bcast_exec() allocates
  * the plan's device tables on a plan's first execution; this call never allocates: it runs the
- * same one-launch WALK kernel, with the tables it needs (tile list, per-chunk hop lists, work
- * counter) placed in a fixed array of BCAST_STATIC_SCRATCH_BYTES bytes that is part of the
+ * same one-launch WALK kernel, with the tables it needs (slice list, per-chunk hop lists and
+ * their offsets) placed in a fixed array of BCAST_STATIC_SCRATCH_BYTES bytes that is part of the
  * library's device image.  Every GPU on which the library is loaded holds that array until the
  * process exits.
  *   rank_bufs, plan, cuda_stream   as for bcast_exec(); inputs and outputs are still the caller's.
  * Behaviour to know about:
- *   - Plans whose tables do not fit (roughly: 24 B per 4..32 KiB tile of the message plus 4 B per
- *     (chunk, message) pair, about 4*P*P bytes) are refused with BCAST_ERR_CAPACITY before
+ *   - Plans whose tables do not fit (roughly: 8 B per slice of the message -- slices are 512 B to
+ *     4 KiB, the larger size is tried before giving up -- plus 4 B per (chunk, message) pair,
+ *     about 4*P*P bytes) are refused with BCAST_ERR_CAPACITY before
  *     anything is copied or launched.  All configurations up to P = 256 ranks with messages up to
  *     512 MiB fit; P = 1024 does not.
  *   - The first call on a device looks up the array's device address (cudaGetSymbolAddress) and
