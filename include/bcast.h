@@ -62,13 +62,12 @@ enum {
 enum {
     /* One launch for the whole plan.  The message is cut into segments on a fixed grid of byte
        offsets (and at chunk boundaries); a warp takes such a slice and carries it through every
-       message of the plan
-       that covers it (scatter hops and ring hops), re-reading it from the source rank's buffer at
-       every hop.  Messages that cover different byte ranges are independent, so no waiting
-       between warps is needed.  The hops of a slice run in an order that respects every `dep`
-       of the plan (no copy is read before the message that delivers it has been performed) but
-       is not the plan's step order where a different order keeps the data in L2: see
-       BCAST_EXEC_WALK_PLAN_ORDER.  Default of bcast_exec(). */
+       message of the plan that covers it (scatter hops and ring hops), re-reading it from the
+       source rank's buffer at every hop.  Messages that cover different byte ranges are
+       independent, so no waiting between warps is needed.  The hops of a slice run in an order
+       that respects every `dep` of the plan (no copy is read before the message that delivers it
+       has been performed) but is not the plan's step order where a different order keeps the
+       data in L2: see BCAST_EXEC_WALK_PLAN_ORDER.  Default of bcast_exec(). */
     BCAST_EXEC_WALK = 0,
     /* One launch per plan step (ceil(log2 P) + P - 1 launches) on the caller's stream; inside a
        launch the messages of that step are cut into tiles and copied in parallel. */
