@@ -177,6 +177,8 @@ def run_ours(args):
     import torch
     import torch.distributed as dist
 
+    from paper_1603_06809_b200.build import ensure_built
+    ensure_built()      # compile the CUDA library if this tree has none yet (atomic replace: safe on every rank)
     from paper_1603_06809_b200 import bcast as B
     from paper_1603_06809_b200 import workloads as W
 

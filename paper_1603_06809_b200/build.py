@@ -39,5 +39,18 @@ def build(force: bool = False, verbose: bool = False) -> str:
     return LIB_PATH
 
 
+def ensure_built() -> str:
+    """Build the library if it is missing; if it is merely older than its sources, try to rebuild
+    and keep the existing one when no compiler is at hand.  Returns the path of the library."""
+    if not os.path.exists(LIB_PATH):
+        return build(force=True)
+    if needs_build():
+        try:
+            return build(force=True)
+        except (OSError, subprocess.CalledProcessError):
+            pass
+    return LIB_PATH
+
+
 if __name__ == "__main__":
     print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))

@@ -10,6 +10,9 @@ if ROOT not in sys.path:
 
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (run with -m gpu on a B200)")
+    # the tests import the ctypes binding at collection time: make sure the library exists
+    from paper_1603_06809_b200.build import ensure_built
+    ensure_built()
 
 
 def golden_path(name: str) -> str:
