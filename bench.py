@@ -51,30 +51,39 @@ def parse_args():
 
 # DRAM bytes of one launch of the dominant kernel (tuned variant), from ncu:
 # dram__bytes_read.sum + dram__bytes_write.sum.  A figure is only valid for the kernel source it
-# was taken with, so each carries the SHA-256 of csrc/exec.cu; once the file changes, `traffic`
-# is reported as null until the counters are taken again.
+# was taken with, so each carries the SHA-256 of the device code in csrc/exec.cu; once that
+# changes, `traffic` is reported as null until the counters are taken again.
 NCU_TRAFFIC = {
     # profiles/bcast_walk_kernel_P100_64MiB_launch_list_and_dram.md
     ("cfg4", "walk"): {"dram_bytes_per_launch": 68298752 + 6586297856,
-                       "exec_cu_sha256": "2b99f7d17361560fd69fbb595060452d5fa3e6d68febc40b046cd653b3041b40"},
+                       "kernel_sha256": "c235a1d6e3b15c2ace154c77f00de995f53e9c7977a640b23b88724310e66f5e"},
     # profiles/bcast_walk_kernel_P64_16MiB_ncu_full.md (same one-pass metric pair, cfg3)
     ("cfg3", "walk"): {"dram_bytes_per_launch": 17127424 + 998557952,
-                       "exec_cu_sha256": "2b99f7d17361560fd69fbb595060452d5fa3e6d68febc40b046cd653b3041b40"},
+                       "kernel_sha256": "c235a1d6e3b15c2ace154c77f00de995f53e9c7977a640b23b88724310e66f5e"},
 }
 
 
-def ncu_traffic(workload, mode):
+KERNEL_BEGIN = "// ---- memory operations."
+KERNEL_END = "// ======================================================================================= host"
+
+
+def kernel_source_sha256():
+    """SHA-256 of the device code of csrc/exec.cu (everything between the two marker comments)."""
     import hashlib
+    path = os.path.join(ROOT, "paper_1603_06809_b200", "csrc", "exec.cu")
+    try:
+        with open(path) as f:
+            text = f.read()
+        return hashlib.sha256(text[text.index(KERNEL_BEGIN):text.index(KERNEL_END)].encode()).hexdigest()
+    except (OSError, ValueError):
+        return None
+
+
+def ncu_traffic(workload, mode):
     rec = NCU_TRAFFIC.get((workload, mode))
     if not rec:
         return None
-    path = os.path.join(ROOT, "paper_1603_06809_b200", "csrc", "exec.cu")
-    try:
-        with open(path, "rb") as f:
-            sha = hashlib.sha256(f.read()).hexdigest()
-    except OSError:
-        return None
-    return rec["dram_bytes_per_launch"] if sha == rec["exec_cu_sha256"] else None
+    return rec["dram_bytes_per_launch"] if kernel_source_sha256() == rec["kernel_sha256"] else None
 
 
 def measured_peak():

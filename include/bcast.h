@@ -156,8 +156,10 @@ uint64_t bcast_plan_total_bytes(const bcast_plan_t *plan);       /* sum of len o
  * outside those ranges has been written.
  * The first execution of a plan allocates and fills the plan's device tables (cudaMalloc and
  * blocking copies); later executions allocate nothing.
- * Errors: BCAST_ERR_INVAL (NULL arguments, NULL/misaligned/overlapping buffers, a device other
- * than the one the plan was first executed on), BCAST_ERR_NOMEM, BCAST_ERR_CUDA.
+ * Errors: BCAST_ERR_INVAL (NULL arguments, NULL/misaligned/overlapping buffers, a buffer that is not
+ * device or managed memory of the current device, a device other than the one the plan was first
+ * executed on), BCAST_ERR_NOMEM, BCAST_ERR_CUDA.  Arguments are checked before anything is
+ * launched; the extent of a buffer cannot be checked.
  */
 int bcast_exec(void *const *rank_bufs, const bcast_plan_t *plan, void *cuda_stream);
 

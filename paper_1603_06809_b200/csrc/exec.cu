@@ -542,13 +542,33 @@ int validate_bufs(void *const *rank_bufs, size_t P, uint64_t nbytes)
     return BCAST_OK;
 }
 
-// The same check, skipped when the pointers are the ones that passed it last time.
+// Every rank buffer must be memory of the current device (or managed memory): a host pointer
+// handed to the kernels would fault the GPU.  Only the first byte of each buffer can be checked.
+int validate_device_memory(void *const *rank_bufs, size_t P)
+{
+    int device = -1;
+    CUDA_TRY(cudaGetDevice(&device));
+    for (size_t k = 0; k < P; k++) {
+        cudaPointerAttributes attr;
+        const cudaError_t e = cudaPointerGetAttributes(&attr, rank_bufs[k]);
+        if (e != cudaSuccess) {
+            cudaGetLastError();   // not a sticky error: clear it
+            return BCAST_ERR_INVAL;
+        }
+        if (attr.type == cudaMemoryTypeManaged) continue;
+        if (attr.type != cudaMemoryTypeDevice || attr.device != device) return BCAST_ERR_INVAL;
+    }
+    return BCAST_OK;
+}
+
+// Both checks, skipped when the pointers are the ones that passed them last time.
 int check_bufs(void *const *rank_bufs, const bcast_plan_t &p, bcast_device_state &ds)
 {
     const size_t P = (size_t)p.P;
     if (ds.checked_bufs.size() == P && std::memcmp(ds.checked_bufs.data(), rank_bufs, P * sizeof(void *)) == 0)
         return BCAST_OK;
-    const int rc = validate_bufs(rank_bufs, P, p.nbytes);
+    int rc = validate_bufs(rank_bufs, P, p.nbytes);
+    if (!rc) rc = validate_device_memory(rank_bufs, P);
     if (rc) return rc;
     ds.checked_bufs.assign(rank_bufs, rank_bufs + P);
     return BCAST_OK;
@@ -757,6 +777,7 @@ constexpr int kMaxDevices = 64;
 std::mutex g_static_mu;
 unsigned char *g_static_addr[kMaxDevices] = {};   // device address of g_static_scratch, per device
 int g_static_sms[kMaxDevices] = {};
+std::vector<void *> g_static_checked;             // rank buffers that last passed the device-memory check
 
 inline size_t round256(size_t x) { return (x + 255) & ~(size_t)255; }
 
@@ -784,6 +805,15 @@ int exec_static(void *const *rank_bufs, const bcast_plan_t &p, cudaStream_t st)
 {
     int rc = validate_bufs(rank_bufs, (size_t)p.P, p.nbytes);
     if (rc) return rc;
+    {
+        // the device-memory check costs a driver call per buffer: remember the last set that passed
+        std::lock_guard<std::mutex> lock(g_static_mu);
+        if (g_static_checked.size() != (size_t)p.P ||
+            std::memcmp(g_static_checked.data(), rank_bufs, (size_t)p.P * sizeof(void *)) != 0) {
+            if ((rc = validate_device_memory(rank_bufs, (size_t)p.P))) return rc;
+            g_static_checked.assign(rank_bufs, rank_bufs + p.P);
+        }
+    }
     if (p.total_bytes == 0) return BCAST_OK;
     unsigned char *scratch = nullptr;
     int sms = 0;

@@ -284,10 +284,14 @@ def test_exec_rejects_bad_buffers():
     bufs = RankBuffers(wl.P, wl.root, wl.nbytes, msg)
     plan = B.bcast_plan(wl.P, wl.root, wl.nbytes, B.BCAST_TUNED)
     good = bufs.pointers()
+    host_pinned = torch.zeros(8192, dtype=torch.uint8).pin_memory()
+    host_plain = np.zeros(8192, dtype=np.uint8)
     for bad in ([good[0], 0, good[2], good[3]],                  # NULL
                 [good[0], good[1] + 8, good[2], good[3]],        # misaligned
                 [good[0], good[1], good[1], good[3]],            # duplicate
-                [good[0], good[0] + 1024, good[2], good[3]]):    # overlapping
+                [good[0], good[0] + 1024, good[2], good[3]],     # overlapping
+                [good[0], host_pinned.data_ptr(), good[2], good[3]],          # pinned host memory
+                [good[0], host_plain.ctypes.data // 16 * 16 + 16, good[2], good[3]]):   # pageable host memory
         with pytest.raises(B.BcastError) as e:
             B.bcast_exec(bad, plan)
         assert e.value.code == B.BCAST_ERR_INVAL

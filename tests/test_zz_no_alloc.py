@@ -56,6 +56,20 @@ def test_static_same_plan_twice_without_reset_between():
     assert all(torch.equal(a, b) for a, b in zip(bufs.view, ref.view))
 
 
+def test_static_refuses_host_memory():
+    wl = W.Workload("static_bad", 4, 0, 4096, 2)
+    bufs = RankBuffers(wl.P, wl.root, wl.nbytes, W.message_bytes(wl.seed, wl.nbytes))
+    plan = B.bcast_plan(wl.P, wl.root, wl.nbytes, B.BCAST_TUNED)
+    good = bufs.pointers()
+    host = torch.zeros(8192, dtype=torch.uint8).pin_memory()
+    with pytest.raises(B.BcastError) as e:
+        B.bcast_exec_static([good[0], host.data_ptr(), good[2], good[3]], plan, torch.cuda.current_stream())
+    assert e.value.code == B.BCAST_ERR_INVAL
+    B.bcast_exec_static(good, plan, torch.cuda.current_stream())
+    torch.cuda.synchronize()
+    assert bufs.all_equal_message() and bufs.guards_intact()
+
+
 def test_static_refuses_plans_beyond_its_capacity():
     P, n = 1024, 64 * 1024
     plan = B.bcast_plan(P, 0, n, B.BCAST_NATIVE)        # about 4 * P * P bytes of hop lists: too large
