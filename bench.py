@@ -2,7 +2,7 @@
 """Benchmark of the scatter-ring-allgather broadcast over P virtual ranks in one GPU's memory.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
-                    [--workload cfg3|cfg4] [--mode walk|walk_plan_order|steps|graph]
+                    [--workload cfg3|cfg4] [--mode walk|walk_plan_order|walk_bulk|auto|steps|graph]
 
 One "step" is one whole broadcast of the tuned variant (binomial scatter + tuned ring allgather,
 every message of the plan) over the workload's P rank buffers.  The headline metric is the
@@ -42,7 +42,7 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg4", choices=["cfg3", "cfg4"])
-    ap.add_argument("--mode", default="walk", choices=["walk", "walk_plan_order", "steps", "graph"])
+    ap.add_argument("--mode", default="walk", choices=["walk", "walk_plan_order", "walk_bulk", "auto", "steps", "graph"])
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-clocks", action="store_true", help="skip the nvidia-smi sampling (profiling runs)")
@@ -203,6 +203,7 @@ def run_ours(args):
 
     wl = {"cfg3": W.CFG3, "cfg4": W.CFG4}[args.workload]
     mode = {"walk": B.BCAST_EXEC_WALK, "walk_plan_order": B.BCAST_EXEC_WALK_PLAN_ORDER,
+            "walk_bulk": B.BCAST_EXEC_WALK_BULK, "auto": B.BCAST_EXEC_AUTO,
             "steps": B.BCAST_EXEC_STEPS, "graph": B.BCAST_EXEC_GRAPH}[args.mode]
     P, n = wl.P, wl.nbytes
     stride = (n + 511) // 256 * 256
@@ -271,7 +272,8 @@ def run_ours(args):
     roofline = {
         "bound": "hbm", "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
         "frac": round(achieved / peak, 4), "traffic": traffic,
-        "kernel": "bcast_walk_kernel" if args.mode.startswith("walk") else "bcast_step_kernel",
+        "kernel": {"walk": "bcast_walk_kernel", "walk_plan_order": "bcast_walk_kernel", "auto": "bcast_walk_kernel",
+                   "walk_bulk": "bcast_walk_bulk_kernel"}.get(args.mode, "bcast_step_kernel"),
         "peak_source": peak_src,
         "algorithmic_bytes_per_launch": alg_bytes_per_launch,
         "launch_ms": round(launch_ms, 5),

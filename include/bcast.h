@@ -55,7 +55,8 @@ enum {
     BCAST_ERR_INVAL = -1,  /* bad argument (range, null, misaligned or overlapping buffers) */
     BCAST_ERR_NOMEM = -2,  /* host or device allocation failed                              */
     BCAST_ERR_CUDA = -3,   /* a CUDA runtime call failed; see bcast_last_cuda_error()       */
-    BCAST_ERR_CAPACITY = -4 /* bcast_exec_static only: the plan's tables exceed the built-in scratch */
+    BCAST_ERR_CAPACITY = -4, /* bcast_exec_static only: the plan's tables exceed the built-in scratch */
+    BCAST_ERR_TIMEOUT = -5   /* bcast_exec_status only: a bounded wait inside a kernel ran out          */
 };
 
 /* How bcast_exec_mode() runs a plan.  All modes perform exactly the plan's messages. */
@@ -67,7 +68,7 @@ enum {
        independent, so no waiting between warps is needed.  The hops of a slice run in an order
        that respects every `dep` of the plan (no copy is read before the message that delivers it
        has been performed) but is not the plan's step order where a different order keeps the
-       data in L2: see BCAST_EXEC_WALK_PLAN_ORDER.  Default of bcast_exec(). */
+       data in L2: see BCAST_EXEC_WALK_PLAN_ORDER. */
     BCAST_EXEC_WALK = 0,
     /* One launch per plan step (ceil(log2 P) + P - 1 launches) on the caller's stream; inside a
        launch the messages of that step are cut into tiles and copied in parallel. */
@@ -77,7 +78,19 @@ enum {
     /* BCAST_EXEC_WALK with the hops of every slice strictly in plan order (all scatter levels,
        then the ring steps in ascending order).  Same copies, same result; in the tuned variant
        the copies the scatter left at inner tree nodes are then re-read from DRAM instead of L2. */
-    BCAST_EXEC_WALK_PLAN_ORDER = 3
+    BCAST_EXEC_WALK_PLAN_ORDER = 3,
+    /* BCAST_EXEC_WALK for large messages, with the data moved by the bulk-copy engine (TMA):
+       whole 16 KiB segments go global -> shared -> global, one worker thread and one mbarrier per
+       segment, twelve segments in flight per SM; segments cut by a chunk boundary are walked through
+       registers as in BCAST_EXEC_WALK.  Same copies, same hop order, same result.  Its waits on the
+       copy engine are bounded: see bcast_exec_status(). */
+    BCAST_EXEC_WALK_BULK = 4,
+    /* The fastest of the above for the plan at hand; what bcast_exec() uses.  BCAST_EXEC_WALK_BULK
+       when the message is too large to be in flight all at once (more than about 1.4 x 32 KB per
+       SM) and the variant is not the tuned one (whose hop order re-reads a segment up to a tree
+       level later, by which time the bulk path's larger working set has left L2); otherwise
+       BCAST_EXEC_WALK. */
+    BCAST_EXEC_AUTO = 5
 };
 
 /* One message of the schedule.  Plain data, 48 bytes, host memory. */
@@ -163,9 +176,9 @@ uint64_t bcast_plan_total_bytes(const bcast_plan_t *plan);       /* sum of len o
  */
 int bcast_exec(void *const *rank_bufs, const bcast_plan_t *plan, void *cuda_stream);
 
-/* bcast_exec with an explicit execution mode (BCAST_EXEC_*); same contract.  BCAST_EXEC_GRAPH
-   captures and instantiates its graph on the first call and again whenever rank_bufs differs
-   from the previous call. */
+/* bcast_exec (which uses BCAST_EXEC_AUTO) with an explicit execution mode; same contract.
+   BCAST_EXEC_GRAPH captures and instantiates its graph on the first call and again whenever
+   rank_bufs differs from the previous call. */
 int bcast_exec_mode(void *const *rank_bufs, const bcast_plan_t *plan, void *cuda_stream, int mode);
 
 /*
@@ -228,6 +241,17 @@ int bcast_exec_static(void *const *rank_bufs, const bcast_plan_t *plan, void *cu
  * (Sections III-A and IV: a process can only pass on what it has received).
  */
 int64_t bcast_plan_walk_order(const bcast_plan_t *plan, int chunk, int mode, int64_t *out, int64_t cap);
+
+/*
+ * bcast_exec_status -- did a kernel of this plan give up on a bounded wait?
+ * The bulk-copy kernel (BCAST_EXEC_WALK_BULK) polls an mbarrier for the arrival of every load; the
+ * number of polls is limited, so that a copy that never completes ends the kernel instead of
+ * hanging the GPU.  A worker whose limit runs out sets a flag in the plan's device state and stops;
+ * the rank buffers are then incomplete.  Call this after the stream has been synchronised: it reads
+ * the flag (a blocking 4-byte copy), clears it, and returns BCAST_ERR_TIMEOUT if it was set, else
+ * BCAST_OK.  The other executors have no waits and never set it.
+ */
+int bcast_exec_status(const bcast_plan_t *plan);
 
 /* Number of kernel launches one execution of the plan enqueues in the given mode (0 if nothing
    has to move); a CUDA-graph replay counts the kernels inside the graph. */

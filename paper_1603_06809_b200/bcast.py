@@ -21,9 +21,10 @@ _lib = ctypes.CDLL(_LIB_PATH)
 BCAST_MAX_RANKS = 1024
 BCAST_NATIVE, BCAST_TUNED, BCAST_DOUBLING = 0, 1, 2
 BCAST_PHASE_SCATTER, BCAST_PHASE_RING = 0, 1
-BCAST_OK, BCAST_ERR_INVAL, BCAST_ERR_NOMEM, BCAST_ERR_CUDA, BCAST_ERR_CAPACITY = 0, -1, -2, -3, -4
+BCAST_OK, BCAST_ERR_INVAL, BCAST_ERR_NOMEM, BCAST_ERR_CUDA, BCAST_ERR_CAPACITY, BCAST_ERR_TIMEOUT = 0, -1, -2, -3, -4, -5
 BCAST_STATIC_SCRATCH_BYTES = 2 << 20
 BCAST_EXEC_WALK, BCAST_EXEC_STEPS, BCAST_EXEC_GRAPH, BCAST_EXEC_WALK_PLAN_ORDER = 0, 1, 2, 3
+BCAST_EXEC_WALK_BULK, BCAST_EXEC_AUTO = 4, 5
 
 #: numpy view of ``bcast_xfer_t`` (48 bytes)
 XFER_DTYPE = np.dtype([
@@ -37,7 +38,7 @@ SYMBOLS = (
     "bcast_plan_nbytes", "bcast_plan_scatter_size", "bcast_plan_num_xfers", "bcast_plan_num_steps",
     "bcast_plan_xfers", "bcast_plan_step_begin", "bcast_plan_bytes_sent", "bcast_plan_bytes_recv",
     "bcast_plan_msgs_sent", "bcast_plan_msgs_recv", "bcast_plan_total_bytes", "bcast_plan_walk_order", "bcast_exec",
-    "bcast_exec_mode", "bcast_exec_host", "bcast_exec_static", "bcast_exec_num_launches", "bcast_strerror",
+    "bcast_exec_mode", "bcast_exec_host", "bcast_exec_static", "bcast_exec_status", "bcast_exec_num_launches", "bcast_strerror",
     "bcast_last_cuda_error",
 )
 
@@ -58,6 +59,7 @@ _sig = {
     "bcast_exec_mode": (_i, [_vpp, _vp, _vp, _i]),
     "bcast_exec_host": (_i, [_vpp, _vp, _vp, _i, _vp, _vpp]),
     "bcast_exec_static": (_i, [_vpp, _vp, _vp]),
+    "bcast_exec_status": (_i, [_vp]),
     "bcast_exec_num_launches": (_i64, [_vp, _i]),
     "bcast_strerror": (ctypes.c_char_p, [_i]),
     "bcast_last_cuda_error": (_i, []),
@@ -235,6 +237,12 @@ def bcast_exec_static(rank_bufs, plan: Plan, stream=None) -> None:
         raise BcastError(BCAST_ERR_INVAL, "bcast_exec_static (len(rank_bufs) != P)")
     _check(_lib.bcast_exec_static(_ptr_array(rank_bufs, "rank_bufs"), plan.handle, _stream_ptr(stream)),
            "bcast_exec_static")
+
+
+def bcast_exec_status(plan: Plan) -> None:
+    """After a stream synchronisation: raises ``BcastError`` (``BCAST_ERR_TIMEOUT``) if a kernel of
+    this plan gave up on one of its bounded waits; returns None otherwise."""
+    _check(_lib.bcast_exec_status(plan.handle), "bcast_exec_status")
 
 
 def bcast_exec_num_launches(plan: Plan, mode: int = BCAST_EXEC_WALK) -> int:

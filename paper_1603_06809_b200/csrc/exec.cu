@@ -121,77 +121,155 @@ __device__ __forceinline__ Split split16(uint64_t lo, uint64_t hi)
 // The (src, dst) pair of hop h+1 is fetched while the loads of hop h are in flight.
 constexpr int kWarpsPerBlock = kThreads / 32;
 
+// One slice, all its hops, by one warp with U words per lane (the register path).
+template <int U, int MAXP>
+__device__ __forceinline__ void walk_slice(const RankPtrs<MAXP> &bufs, const WalkSlice sl, uint64_t scatter_size,
+                                           uint64_t nbytes, const uint32_t *__restrict__ hops,
+                                           const int *__restrict__ hop_begin, uint32_t lane)
+{
+    constexpr uint64_t kSeg = 32ull * U * 16;
+    const uint64_t seg_lo = (uint64_t)sl.seg * kSeg, seg_hi = seg_lo + kSeg;
+    const uint64_t lo = max(min((uint64_t)sl.chunk * scatter_size, nbytes), seg_lo);
+    const uint64_t hi = min(min(((uint64_t)sl.chunk + 1) * scatter_size, nbytes), seg_hi);
+    if (lo >= hi) return;
+    const uint32_t *hp = hops + hop_begin[sl.chunk];
+    const int nh = hop_begin[sl.chunk + 1] - hop_begin[sl.chunk];
+    if (nh <= 0) return;
+    const uint64_t base = seg_lo + (uint64_t)lane * 16;
+
+    uint32_t e = __ldg(hp);
+    const uint8_t *s = bufs.p[e & 0xffffu];
+    uint8_t *d = bufs.p[e >> 16];
+    if (lo == seg_lo && hi == seg_hi) {
+        // whole segment: every lane moves U words per hop, no predicates
+        for (int h = 0; h < nh; h++) {
+            uint4 v[U];
+#pragma unroll
+            for (int u = 0; u < U; u++) v[u] = ld16(s + base + (uint64_t)u * 512);
+            e = __ldg(hp + min(h + 1, nh - 1));              // next hop, while the loads are in flight
+            const uint8_t *s_next = bufs.p[e & 0xffffu];
+            uint8_t *d_next = bufs.p[e >> 16];
+#pragma unroll
+            for (int u = 0; u < U; u++) st16(d + base + (uint64_t)u * 512, v[u]);
+            s = s_next;
+            d = d_next;
+        }
+    } else {
+        // ragged slice (a chunk starts or ends inside the segment): predicated words, plus the
+        // bytes of the partial words at either end
+        const uint64_t body_lo = (lo + 15) & ~(uint64_t)15, body_hi = hi & ~(uint64_t)15;
+        const uint64_t head_end = body_lo < hi ? body_lo : hi;
+        const uint64_t tail_begin = body_hi > head_end ? body_hi : head_end;
+        const uint32_t nhead = (uint32_t)(head_end - lo), nedge = nhead + (uint32_t)(hi - tail_begin);
+        bool ok[U];
+#pragma unroll
+        for (int u = 0; u < U; u++) {
+            const uint64_t o = base + (uint64_t)u * 512;
+            ok[u] = o >= body_lo && o + 16 <= body_hi;
+        }
+        const bool has_edge = lane < nedge;
+        const uint64_t eoff = lane < nhead ? lo + lane : tail_begin + (lane - nhead);
+        for (int h = 0; h < nh; h++) {
+            uint4 v[U];
+            uint32_t b = 0;
+#pragma unroll
+            for (int u = 0; u < U; u++)
+                if (ok[u]) v[u] = ld16(s + base + (uint64_t)u * 512);
+            if (has_edge) b = ld1(s + eoff);
+            e = __ldg(hp + min(h + 1, nh - 1));
+            const uint8_t *s_next = bufs.p[e & 0xffffu];
+            uint8_t *d_next = bufs.p[e >> 16];
+#pragma unroll
+            for (int u = 0; u < U; u++)
+                if (ok[u]) st16(d + base + (uint64_t)u * 512, v[u]);
+            if (has_edge) st1(d + eoff, b);
+            s = s_next;
+            d = d_next;
+        }
+    }
+}
+
 template <int U, int MAXP>
 __global__ void __launch_bounds__(kThreads)
 bcast_walk_kernel(const __grid_constant__ RankPtrs<MAXP> bufs, const WalkSlice *__restrict__ slices,
                   long long n_slices, uint64_t scatter_size, uint64_t nbytes,
                   const uint32_t *__restrict__ hops, const int *__restrict__ hop_begin)
 {
-    constexpr uint64_t kSeg = 32ull * U * 16;
     const uint32_t lane = threadIdx.x & 31u;
     const long long total_warps = (long long)gridDim.x * kWarpsPerBlock;
-
     // slice w goes to block w mod gridDim.x: every SM gets the same number of slices (+-1)
-    for (long long w = (long long)(threadIdx.x >> 5) * gridDim.x + blockIdx.x; w < n_slices; w += total_warps) {
-        const WalkSlice sl = slices[w];
-        const uint64_t seg_lo = (uint64_t)sl.seg * kSeg, seg_hi = seg_lo + kSeg;
-        const uint64_t lo = max(min((uint64_t)sl.chunk * scatter_size, nbytes), seg_lo);
-        const uint64_t hi = min(min(((uint64_t)sl.chunk + 1) * scatter_size, nbytes), seg_hi);
-        if (lo >= hi) continue;
+    for (long long w = (long long)(threadIdx.x >> 5) * gridDim.x + blockIdx.x; w < n_slices; w += total_warps)
+        walk_slice<U, MAXP>(bufs, slices[w], scatter_size, nbytes, hops, hop_begin, lane);
+}
+
+// ------------------------------------------------------------------------------------- WALK, bulk copies
+// The same walk for large messages, with the data moved by the bulk-copy engine (TMA, untiled
+// cp.async.bulk) instead of through registers: whole 16 KiB segments of the fixed grid go
+// global -> shared -> global, one worker thread per segment.  A hop is: expect 16 KiB on the
+// worker's mbarrier, bulk load from the source rank's buffer, wait, bulk store to the destination
+// rank's buffer, wait until the store has completed (not merely been read out of shared memory:
+// the next hop may load those very bytes again).  Two memory round trips per hop instead of one
+// are paid for with more bytes in flight (kBulkWorkers x 16 KiB per block); the longer contiguous
+// runs are what DRAM likes better.  Segments that a chunk boundary cuts are left to a second warp
+// of every block, which walks them as 4 KiB register slices.
+// Every address and size handed to a bulk copy is a multiple of 16 bytes (rank buffers are
+// 16-byte aligned, segment offsets and sizes are multiples of 16 KiB).  No cluster multicast.
+constexpr uint32_t kBulkSeg = 16384;
+constexpr int kBulkWorkers = 4;               // worker threads (lanes 0..3 of warp 0) and segments in flight per block
+constexpr int kBulkThreads = 64;              // warp 0: bulk workers; warp 1: register slices
+constexpr int kBulkSpinLimit = 1 << 24;       // mbarrier polls before a worker gives up
+
+template <int MAXP>
+__global__ void __launch_bounds__(kBulkThreads)
+bcast_walk_bulk_kernel(const __grid_constant__ RankPtrs<MAXP> bufs, const WalkSlice *__restrict__ bulk_slices,
+                       long long n_bulk, const WalkSlice *__restrict__ reg_slices, long long n_reg,
+                       uint64_t scatter_size, uint64_t nbytes, const uint32_t *__restrict__ hops,
+                       const int *__restrict__ hop_begin, int *status)
+{
+    extern __shared__ __align__(128) uint8_t bulk_smem[];
+    __shared__ __align__(8) uint64_t bulk_bar[kBulkWorkers];
+    const uint32_t lane = threadIdx.x & 31u;
+
+    if (threadIdx.x >= 32) {
+        // warp 1: the segments cut by chunk boundaries, as register slices of 8 words per lane
+        for (long long w = blockIdx.x; w < n_reg; w += gridDim.x)
+            walk_slice<8, MAXP>(bufs, reg_slices[w], scatter_size, nbytes, hops, hop_begin, lane);
+        return;
+    }
+    if (lane >= kBulkWorkers) return;
+
+    const uint32_t sbuf = (uint32_t)__cvta_generic_to_shared(bulk_smem + (size_t)lane * kBulkSeg);
+    const uint32_t sbar = (uint32_t)__cvta_generic_to_shared(&bulk_bar[lane]);
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" :: "r"(sbar) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    uint32_t phase = 0;
+    const long long total = (long long)gridDim.x * kBulkWorkers;
+    for (long long w = (long long)lane * gridDim.x + blockIdx.x; w < n_bulk; w += total) {
+        const WalkSlice sl = bulk_slices[w];
+        const uint64_t off = (uint64_t)sl.seg * kBulkSeg;
         const uint32_t *hp = hops + hop_begin[sl.chunk];
         const int nh = hop_begin[sl.chunk + 1] - hop_begin[sl.chunk];
-        if (nh <= 0) continue;
-        const uint64_t base = seg_lo + (uint64_t)lane * 16;
-
-        uint32_t e = __ldg(hp);
-        const uint8_t *s = bufs.p[e & 0xffffu];
-        uint8_t *d = bufs.p[e >> 16];
-        if (lo == seg_lo && hi == seg_hi) {
-            // whole segment: every lane moves U words per hop, no predicates
-            for (int h = 0; h < nh; h++) {
-                uint4 v[U];
-#pragma unroll
-                for (int u = 0; u < U; u++) v[u] = ld16(s + base + (uint64_t)u * 512);
-                e = __ldg(hp + min(h + 1, nh - 1));              // next hop, while the loads are in flight
-                const uint8_t *s_next = bufs.p[e & 0xffffu];
-                uint8_t *d_next = bufs.p[e >> 16];
-#pragma unroll
-                for (int u = 0; u < U; u++) st16(d + base + (uint64_t)u * 512, v[u]);
-                s = s_next;
-                d = d_next;
+        for (int h = 0; h < nh; h++) {
+            const uint32_t e = __ldg(hp + h);
+            const uint8_t *s = bufs.p[e & 0xffffu] + off;
+            uint8_t *d = bufs.p[e >> 16] + off;
+            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(sbar), "r"(kBulkSeg) : "memory");
+            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                         :: "r"(sbuf), "l"(s), "r"(kBulkSeg), "r"(sbar) : "memory");
+            uint32_t arrived = 0;
+            for (int spin = 0; spin < kBulkSpinLimit && !arrived; spin++)
+                asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+                             : "=r"(arrived) : "r"(sbar), "r"(phase) : "memory");
+            if (!arrived) {
+                // the load never reported completion: flag it for the host and stop this worker
+                // (nothing else of this worker is in flight: its last store was waited for)
+                atomicExch(status, 1);
+                return;
             }
-        } else {
-            // ragged slice (a chunk starts or ends inside the segment): predicated words, plus the
-            // bytes of the partial words at either end
-            const uint64_t body_lo = (lo + 15) & ~(uint64_t)15, body_hi = hi & ~(uint64_t)15;
-            const uint64_t head_end = body_lo < hi ? body_lo : hi;
-            const uint64_t tail_begin = body_hi > head_end ? body_hi : head_end;
-            const uint32_t nhead = (uint32_t)(head_end - lo), nedge = nhead + (uint32_t)(hi - tail_begin);
-            bool ok[U];
-#pragma unroll
-            for (int u = 0; u < U; u++) {
-                const uint64_t o = base + (uint64_t)u * 512;
-                ok[u] = o >= body_lo && o + 16 <= body_hi;
-            }
-            const bool has_edge = lane < nedge;
-            const uint64_t eoff = lane < nhead ? lo + lane : tail_begin + (lane - nhead);
-            for (int h = 0; h < nh; h++) {
-                uint4 v[U];
-                uint32_t b = 0;
-#pragma unroll
-                for (int u = 0; u < U; u++)
-                    if (ok[u]) v[u] = ld16(s + base + (uint64_t)u * 512);
-                if (has_edge) b = ld1(s + eoff);
-                e = __ldg(hp + min(h + 1, nh - 1));
-                const uint8_t *s_next = bufs.p[e & 0xffffu];
-                uint8_t *d_next = bufs.p[e >> 16];
-#pragma unroll
-                for (int u = 0; u < U; u++)
-                    if (ok[u]) st16(d + base + (uint64_t)u * 512, v[u]);
-                if (has_edge) st1(d + eoff, b);
-                s = s_next;
-                d = d_next;
-            }
+            phase ^= 1u;
+            asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" :: "l"(d), "r"(sbuf), "r"(kBulkSeg) : "memory");
+            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+            asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
         }
     }
 }
@@ -252,6 +330,12 @@ struct bcast_device_state {
     int *d_hop_begin = nullptr;
     long long n_slices = 0;
     int walk_u = 0, walk_grid = 0;
+    bool bandwidth_regime = false;     // message too large to be in flight at once
+    // WALK with bulk copies
+    WalkSlice *d_bulk_slices = nullptr, *d_reg_slices = nullptr;
+    long long n_bulk = 0, n_reg = 0;
+    int bulk_grid = 0;
+    int *d_status = nullptr;           // set by a kernel whose bounded wait ran out
     // argument check cache
     std::vector<void *> checked_bufs;
 };
@@ -266,6 +350,9 @@ void bcast_device_state_free(bcast_device_state *dev)
     if (dev->graph) cudaGraphDestroy(dev->graph);
     cudaFree(dev->d_xfers);
     cudaFree(dev->d_slices);
+    cudaFree(dev->d_bulk_slices);
+    cudaFree(dev->d_reg_slices);
+    cudaFree(dev->d_status);
     cudaFree(dev->d_hops);
     cudaFree(dev->d_hops_plan);
     cudaFree(dev->d_hop_begin);
@@ -445,6 +532,7 @@ int walk_blocks_per_sm(int u, int P, int *bps)
 // BCAST_WALK_WORDS and BCAST_WALK_BLOCKS_PER_SM override the choice (for experiments).
 struct WalkShape {
     int u = 1, grid = 1;
+    bool bandwidth_regime = false;
 };
 
 int choose_walk_shape(const bcast_plan_t &p, int sm_count, WalkShape *shape)
@@ -464,6 +552,7 @@ int choose_walk_shape(const bcast_plan_t &p, int sm_count, WalkShape *shape)
     } else if (count_walk_slices(p, 8) * 5 > (long long)sm_count * kWarpsPerBlock * 7) {   // > 1.4 rounds
         u = 8;
         bps = 1;
+        shape->bandwidth_regime = true;
     } else {
         for (int cand : {1, 2, 4, 8}) {
             if ((rc = walk_blocks_per_sm(cand, p.P, &resident))) return rc;
@@ -483,6 +572,55 @@ int choose_walk_shape(const bcast_plan_t &p, int sm_count, WalkShape *shape)
     return BCAST_OK;
 }
 
+// Slices of the bulk-copy walk: every whole 16 KiB segment that lies inside one chunk is a bulk
+// slice; what is left of the segments that a chunk boundary (or the end of the message) cuts
+// becomes register slices on the 4 KiB grid of walk_slice<8>.
+void make_bulk_slices(const bcast_plan_t &p, std::vector<WalkSlice> &bulk, std::vector<WalkSlice> &reg)
+{
+    constexpr uint64_t kReg = 32ull * 8 * 16;
+    bulk.clear();
+    reg.clear();
+    for (int c = 0; c < p.P; c++) {
+        const uint64_t b = std::min<uint64_t>((uint64_t)c * p.S, p.nbytes);
+        const uint64_t e = std::min<uint64_t>((uint64_t)(c + 1) * p.S, p.nbytes);
+        for (uint64_t g = b / kBulkSeg; b < e && g * kBulkSeg < e; g++) {
+            const uint64_t lo = std::max(b, g * kBulkSeg), hi = std::min(e, (g + 1) * kBulkSeg);
+            if (hi - lo == kBulkSeg) {
+                bulk.push_back(WalkSlice{(uint32_t)g, (uint32_t)c});
+                continue;
+            }
+            for (uint64_t q = lo / kReg; q * kReg < hi; q++) reg.push_back(WalkSlice{(uint32_t)q, (uint32_t)c});
+        }
+    }
+}
+
+int build_bulk_tables(const bcast_plan_t &p, bcast_device_state &ds)
+{
+    std::vector<WalkSlice> bulk, reg;
+    make_bulk_slices(p, bulk, reg);
+    ds.n_bulk = (long long)bulk.size();
+    ds.n_reg = (long long)reg.size();
+    int rc;
+    if ((rc = upload(&ds.d_bulk_slices, bulk))) return rc;
+    if ((rc = upload(&ds.d_reg_slices, reg))) return rc;
+    CUDA_TRY(cudaMalloc((void **)&ds.d_status, sizeof(int)));
+    CUDA_TRY(cudaMemset(ds.d_status, 0, sizeof(int)));
+    // three blocks of four workers per SM: 192 KB of segments in flight per SM
+    const size_t smem = (size_t)kBulkWorkers * kBulkSeg;
+    int resident = 0;
+    if (p.P <= 128) {
+        CUDA_TRY(cudaFuncSetAttribute(bcast_walk_bulk_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&resident, bcast_walk_bulk_kernel<128>, kBulkThreads, smem));
+    } else {
+        CUDA_TRY(cudaFuncSetAttribute(bcast_walk_bulk_kernel<BCAST_MAX_RANKS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&resident, bcast_walk_bulk_kernel<BCAST_MAX_RANKS>, kBulkThreads, smem));
+    }
+    const int bps = std::max(1, std::min(resident, env_int("BCAST_BULK_BLOCKS_PER_SM", 3)));
+    const long long want = std::max<long long>(1, std::max((ds.n_bulk + kBulkWorkers - 1) / kBulkWorkers, ds.n_reg));
+    ds.bulk_grid = (int)std::min<long long>(want, (long long)ds.sm_count * bps);
+    return BCAST_OK;
+}
+
 // Device tables of the WALK executor, cached in the plan's device state.
 int build_walk_tables(const bcast_plan_t &p, bcast_device_state &ds)
 {
@@ -491,6 +629,7 @@ int build_walk_tables(const bcast_plan_t &p, bcast_device_state &ds)
     if (rc) return rc;
     ds.walk_u = shape.u;
     ds.walk_grid = shape.grid;
+    ds.bandwidth_regime = shape.bandwidth_regime;
     WalkTables t;
     if ((rc = make_walk_tables(p, ds.walk_u, t))) return rc;
     ds.n_slices = (long long)t.slices.size();
@@ -519,6 +658,7 @@ int get_state(const bcast_plan_t &p, bcast_device_state **out)
     try {
         if (!rc) rc = build_step_tables(p, *ds);
         if (!rc) rc = build_walk_tables(p, *ds);
+        if (!rc) rc = build_bulk_tables(p, *ds);
     } catch (const std::bad_alloc &) {
         rc = BCAST_ERR_NOMEM;
     }
@@ -619,6 +759,23 @@ int launch_walk(const bcast_plan_t &p, const bcast_device_state &ds, void *const
 }
 
 template <int MAXP>
+int launch_walk_bulk_tables(const bcast_plan_t &p, const bcast_device_state &ds, void *const *rank_bufs, cudaStream_t st)
+{
+    RankPtrs<MAXP> rp;
+    fill_ptrs(rp, rank_bufs, p.P);
+    bcast_walk_bulk_kernel<MAXP><<<ds.bulk_grid, kBulkThreads, (size_t)kBulkWorkers * kBulkSeg, st>>>(
+        rp, ds.d_bulk_slices, ds.n_bulk, ds.d_reg_slices, ds.n_reg, p.S, p.nbytes, ds.d_hops, ds.d_hop_begin, ds.d_status);
+    CUDA_TRY(cudaGetLastError());
+    return BCAST_OK;
+}
+
+int launch_walk_bulk(const bcast_plan_t &p, const bcast_device_state &ds, void *const *rank_bufs, cudaStream_t st)
+{
+    return p.P <= 128 ? launch_walk_bulk_tables<128>(p, ds, rank_bufs, st)
+                      : launch_walk_bulk_tables<BCAST_MAX_RANKS>(p, ds, rank_bufs, st);
+}
+
+template <int MAXP>
 int launch_steps(const bcast_device_state &ds, void *const *rank_bufs, int P, cudaStream_t st)
 {
     RankPtrs<MAXP> rp;
@@ -664,7 +821,7 @@ int bcast_exec_mode(void *const *rank_bufs, const bcast_plan_t *plan, void *cuda
 {
     if (!rank_bufs || !plan) return BCAST_ERR_INVAL;
     if (mode != BCAST_EXEC_WALK && mode != BCAST_EXEC_STEPS && mode != BCAST_EXEC_GRAPH &&
-        mode != BCAST_EXEC_WALK_PLAN_ORDER)
+        mode != BCAST_EXEC_WALK_PLAN_ORDER && mode != BCAST_EXEC_WALK_BULK && mode != BCAST_EXEC_AUTO)
         return BCAST_ERR_INVAL;
     const bcast_plan_t &p = *plan;
     bcast_device_state *ds = nullptr;
@@ -679,7 +836,15 @@ int bcast_exec_mode(void *const *rank_bufs, const bcast_plan_t *plan, void *cuda
     if (p.total_bytes == 0) return BCAST_OK;   // P = 1 or an empty message: nothing moves
     cudaStream_t st = (cudaStream_t)cuda_stream;
     const int P = p.P;
+    // The bulk-copy walk needs ~4x the bytes in flight of the register walk.  With plan-order hops
+    // (native, doubling) a segment is re-read on the very next hop and that still fits in L2; with
+    // the tuned variant's level-order hops the re-read comes up to a tree level later and no longer
+    // does (measured: 11-20 % slower than the register walk), so the tuned variant stays with registers.
+    if (mode == BCAST_EXEC_AUTO)
+        mode = ds->bandwidth_regime && p.variant != BCAST_TUNED ? BCAST_EXEC_WALK_BULK : BCAST_EXEC_WALK;
     switch (mode) {
+    case BCAST_EXEC_WALK_BULK:
+        return launch_walk_bulk(p, *ds, rank_bufs, st);
     case BCAST_EXEC_WALK:
     case BCAST_EXEC_WALK_PLAN_ORDER: {
         return launch_walk(p, *ds, rank_bufs, mode == BCAST_EXEC_WALK_PLAN_ORDER, st);
@@ -697,7 +862,7 @@ int bcast_exec_mode(void *const *rank_bufs, const bcast_plan_t *plan, void *cuda
 
 int bcast_exec(void *const *rank_bufs, const bcast_plan_t *plan, void *cuda_stream)
 {
-    return bcast_exec_mode(rank_bufs, plan, cuda_stream, BCAST_EXEC_WALK);
+    return bcast_exec_mode(rank_bufs, plan, cuda_stream, BCAST_EXEC_AUTO);
 }
 
 int bcast_exec_host(void *const *rank_bufs, const bcast_plan_t *plan, void *cuda_stream, int mode,
@@ -748,7 +913,9 @@ int64_t bcast_plan_walk_order(const bcast_plan_t *plan, int chunk, int mode, int
 int64_t bcast_exec_num_launches(const bcast_plan_t *plan, int mode)
 {
     if (!plan || plan->total_bytes == 0) return 0;
-    if (mode == BCAST_EXEC_WALK || mode == BCAST_EXEC_WALK_PLAN_ORDER) return 1;
+    if (mode == BCAST_EXEC_WALK || mode == BCAST_EXEC_WALK_PLAN_ORDER || mode == BCAST_EXEC_WALK_BULK ||
+        mode == BCAST_EXEC_AUTO)
+        return 1;
     if (mode != BCAST_EXEC_STEPS && mode != BCAST_EXEC_GRAPH) return 0;
     // a step launches a kernel unless all of its messages are empty
     int64_t n = 0;
@@ -759,6 +926,17 @@ int64_t bcast_exec_num_launches(const bcast_plan_t *plan, int mode)
         n += any;
     }
     return n;
+}
+
+int bcast_exec_status(const bcast_plan_t *plan)
+{
+    if (!plan) return BCAST_ERR_INVAL;
+    if (!plan->dev || !plan->dev->d_status) return BCAST_OK;     // never executed: nothing to report
+    int flag = 0;
+    CUDA_TRY(cudaMemcpy(&flag, plan->dev->d_status, sizeof(int), cudaMemcpyDeviceToHost));
+    if (!flag) return BCAST_OK;
+    CUDA_TRY(cudaMemset(plan->dev->d_status, 0, sizeof(int)));
+    return BCAST_ERR_TIMEOUT;
 }
 
 int bcast_last_cuda_error(void) { return t_last_cuda_error; }

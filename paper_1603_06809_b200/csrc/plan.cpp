@@ -218,6 +218,7 @@ const char *bcast_strerror(int code)
     case BCAST_ERR_NOMEM: return "out of memory";
     case BCAST_ERR_CUDA: return "CUDA runtime error";
     case BCAST_ERR_CAPACITY: return "plan tables exceed the built-in scratch of bcast_exec_static";
+    case BCAST_ERR_TIMEOUT: return "a bounded wait inside a kernel ran out";
     default: return "unknown error code";
     }
 }

@@ -1,6 +1,6 @@
 """Time the native and the tuned broadcast over a set of workloads on one GPU and print a table.
 
-    python -m paper_1603_06809_b200.sweep [--set config5|paper|configs] [--mode walk|walk_plan_order|steps|graph]
+    python -m paper_1603_06809_b200.sweep [--set config5|paper|configs] [--mode auto|walk|walk_plan_order|walk_bulk|steps|graph]
                                            [--iters N] [--json]
 
 For every workload: median time of the tuned and of the native variant (and, where P is a power of
@@ -21,6 +21,7 @@ from . import bcast as B
 from . import workloads as W
 
 MODES = {"walk": B.BCAST_EXEC_WALK, "walk_plan_order": B.BCAST_EXEC_WALK_PLAN_ORDER,
+         "walk_bulk": B.BCAST_EXEC_WALK_BULK, "auto": B.BCAST_EXEC_AUTO,
          "steps": B.BCAST_EXEC_STEPS, "graph": B.BCAST_EXEC_GRAPH}
 
 
@@ -76,7 +77,7 @@ def run(workloads, mode: int, iters: int):
 def main():
     ap = argparse.ArgumentParser(description=__doc__.split("\n")[0])
     ap.add_argument("--set", default="paper", choices=["config5", "paper", "configs"])
-    ap.add_argument("--mode", default="walk", choices=sorted(MODES))
+    ap.add_argument("--mode", default="auto", choices=sorted(MODES))
     ap.add_argument("--iters", type=int, default=50)
     ap.add_argument("--json", action="store_true", help="one JSON object per line instead of a table")
     args = ap.parse_args()

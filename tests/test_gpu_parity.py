@@ -15,8 +15,9 @@ from gpu_harness import RankBuffers, run_broadcast
 
 pytestmark = pytest.mark.gpu
 
-MODES = [B.BCAST_EXEC_WALK, B.BCAST_EXEC_STEPS, B.BCAST_EXEC_GRAPH, B.BCAST_EXEC_WALK_PLAN_ORDER]
-MODE_IDS = ["walk", "steps", "graph", "walk_plan_order"]
+MODES = [B.BCAST_EXEC_WALK, B.BCAST_EXEC_STEPS, B.BCAST_EXEC_GRAPH, B.BCAST_EXEC_WALK_PLAN_ORDER,
+         B.BCAST_EXEC_WALK_BULK, B.BCAST_EXEC_AUTO]
+MODE_IDS = ["walk", "steps", "graph", "walk_plan_order", "walk_bulk", "auto"]
 VARIANTS = [B.BCAST_NATIVE, B.BCAST_TUNED]
 VARIANT_IDS = ["native", "tuned"]
 
@@ -24,6 +25,7 @@ VARIANT_IDS = ["native", "tuned"]
 def check_against_oracle(oracle, wl, variant, mode, shift=0, repeats=1):
     msg = W.message_bytes(wl.seed, wl.nbytes)
     plan, bufs = run_broadcast(wl.P, wl.root, wl.nbytes, variant, mode, msg, shift=shift, repeats=repeats)
+    B.bcast_exec_status(plan)                       # no bounded wait ran out
     ref = oracle.simulate(wl.P, wl.root, wl.nbytes, variant, message=msg)
     got = bufs.to_host()
     assert got.shape == ref.bufs.shape
@@ -113,8 +115,13 @@ def test_runs_on_a_side_stream(oracle):
 def test_cfg4_full_size(oracle, variant):
     wl = W.CFG4
     msg = W.message_bytes(wl.seed, wl.nbytes)
-    plan, bufs = run_broadcast(wl.P, wl.root, wl.nbytes, variant, B.BCAST_EXEC_WALK, msg)
-    assert bufs.all_equal_message() and bufs.guards_intact()
+    for mode in (B.BCAST_EXEC_WALK, B.BCAST_EXEC_AUTO):         # AUTO is the bulk-copy kernel at this size
+        plan, bufs = run_broadcast(wl.P, wl.root, wl.nbytes, variant, mode, msg)
+        assert bufs.all_equal_message() and bufs.guards_intact()
+        B.bcast_exec_status(plan)
+        if mode == B.BCAST_EXEC_WALK:
+            del bufs
+            torch.cuda.empty_cache()
     ref = oracle.simulate(wl.P, wl.root, wl.nbytes, variant, message=msg)
     for k in (0, 1, 37, 62, 63, 64, 99):
         assert np.array_equal(bufs.view[k].cpu().numpy(), ref.bufs[k])
@@ -140,8 +147,9 @@ def test_sweep(oracle, variant):
             check_against_oracle(oracle, wl, variant, B.BCAST_EXEC_WALK)
         else:
             msg = W.message_bytes(wl.seed, wl.nbytes)
-            plan, bufs = run_broadcast(wl.P, wl.root, wl.nbytes, variant, B.BCAST_EXEC_WALK, msg)
+            plan, bufs = run_broadcast(wl.P, wl.root, wl.nbytes, variant, B.BCAST_EXEC_AUTO, msg)
             assert bufs.all_equal_message() and bufs.guards_intact(), wl.name
+            B.bcast_exec_status(plan)
             ref = oracle.simulate(wl.P, wl.root, wl.nbytes, variant)          # schedule and counters only
             assert B.bcast_plan_total_bytes(plan) == int(ref.col("len").sum())
             del bufs
@@ -199,7 +207,7 @@ def test_message_larger_than_4_gib(oracle):
     bufs = [torch.full((n + 512,), 0xC3, dtype=torch.uint8, device="cuda:0") for _ in range(P)]
     views = [b[256:256 + n] for b in bufs]
     views[root].copy_(msg)
-    for mode in (B.BCAST_EXEC_WALK, B.BCAST_EXEC_STEPS):
+    for mode in (B.BCAST_EXEC_WALK, B.BCAST_EXEC_STEPS, B.BCAST_EXEC_WALK_BULK):
         for k in range(P):
             if k != root:
                 views[k].fill_(W.poison_byte(k))

@@ -139,6 +139,10 @@ def test_exec_argument_errors_need_no_gpu():
     assert B._lib.bcast_exec_mode((ctypes.c_void_p * 4)(16, 32, 48, 64), plan.handle, None, 7) == B.BCAST_ERR_INVAL
     assert B.bcast_exec_num_launches(plan, B.BCAST_EXEC_WALK) == 1
     assert B.bcast_exec_num_launches(plan, B.BCAST_EXEC_WALK_PLAN_ORDER) == 1
+    assert B.bcast_exec_num_launches(plan, B.BCAST_EXEC_WALK_BULK) == 1
+    assert B.bcast_exec_num_launches(plan, B.BCAST_EXEC_AUTO) == 1
+    B.bcast_exec_status(plan)                                  # never executed: nothing to report
+    assert B._lib.bcast_exec_status(None) == B.BCAST_ERR_INVAL
     assert B.bcast_exec_num_launches(plan, B.BCAST_EXEC_STEPS) == 2 + 3
     assert B.bcast_exec_num_launches(B.bcast_plan(1, 0, 64, 1), B.BCAST_EXEC_WALK) == 0
     assert B.bcast_exec_num_launches(B.bcast_plan(4, 0, 0, 1), B.BCAST_EXEC_STEPS) == 0
