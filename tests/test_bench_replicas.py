@@ -12,6 +12,13 @@ import torch.multiprocessing as mp
 from helpers import ROOT
 
 
+def _free_port():
+    import socket
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
 def _rank_main(rank, world, port, out):
     import torch.distributed as dist
     sys.path.insert(0, ROOT)
@@ -29,7 +36,7 @@ def _rank_main(rank, world, port, out):
 def test_max_over_ranks_and_whole_job_rate_two_gloo_ranks():
     ctx = mp.get_context("spawn")
     out = ctx.Queue()
-    world, port = 2, 29731
+    world, port = 2, _free_port()
     procs = [ctx.Process(target=_rank_main, args=(r, world, port, out)) for r in range(world)]
     for p in procs:
         p.start()
@@ -53,7 +60,7 @@ def test_reference_arm_under_torchrun_only_rank0_reports():
     """`bench.py --impl reference` launched as two ranks: rank 0 times the CPU oracle and prints the
     one JSON line, the other rank exits 0 without work."""
     cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", "2",
-           "--master-addr", "127.0.0.1", "--master-port", "29733",
+           "--master-addr", "127.0.0.1", "--master-port", str(_free_port()),
            os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2", "--workload", "cfg3",
            "--steps", "1", "--warmup", "0"]
     res = subprocess.run(cmd, capture_output=True, text=True, timeout=600, cwd=ROOT)
