@@ -86,8 +86,8 @@ enum {
        copy engine are bounded: see bcast_exec_status(). */
     BCAST_EXEC_WALK_BULK = 4,
     /* The fastest of the above for the plan at hand; what bcast_exec() uses.  BCAST_EXEC_WALK_BULK
-       when the message is too large to be in flight all at once (more than about 1.4 x 32 KB per
-       SM) and the variant is not the tuned one (whose hop order re-reads a segment up to a tree
+       when the message gives the bulk walk at least two rounds of work (about 58 MB on 148 SMs)
+       and the variant is not the tuned one (whose hop order re-reads a segment up to a tree
        level later, by which time the bulk path's larger working set has left L2); otherwise
        BCAST_EXEC_WALK. */
     BCAST_EXEC_AUTO = 5

@@ -330,7 +330,6 @@ struct bcast_device_state {
     int *d_hop_begin = nullptr;
     long long n_slices = 0;
     int walk_u = 0, walk_grid = 0;
-    bool bandwidth_regime = false;     // message too large to be in flight at once
     // WALK with bulk copies
     WalkSlice *d_bulk_slices = nullptr, *d_reg_slices = nullptr;
     long long n_bulk = 0, n_reg = 0;
@@ -532,7 +531,6 @@ int walk_blocks_per_sm(int u, int P, int *bps)
 // BCAST_WALK_WORDS and BCAST_WALK_BLOCKS_PER_SM override the choice (for experiments).
 struct WalkShape {
     int u = 1, grid = 1;
-    bool bandwidth_regime = false;
 };
 
 int choose_walk_shape(const bcast_plan_t &p, int sm_count, WalkShape *shape)
@@ -552,7 +550,6 @@ int choose_walk_shape(const bcast_plan_t &p, int sm_count, WalkShape *shape)
     } else if (count_walk_slices(p, 8) * 5 > (long long)sm_count * kWarpsPerBlock * 7) {   // > 1.4 rounds
         u = 8;
         bps = 1;
-        shape->bandwidth_regime = true;
     } else {
         for (int cand : {1, 2, 4, 8}) {
             if ((rc = walk_blocks_per_sm(cand, p.P, &resident))) return rc;
@@ -629,7 +626,6 @@ int build_walk_tables(const bcast_plan_t &p, bcast_device_state &ds)
     if (rc) return rc;
     ds.walk_u = shape.u;
     ds.walk_grid = shape.grid;
-    ds.bandwidth_regime = shape.bandwidth_regime;
     WalkTables t;
     if ((rc = make_walk_tables(p, ds.walk_u, t))) return rc;
     ds.n_slices = (long long)t.slices.size();
@@ -840,8 +836,12 @@ int bcast_exec_mode(void *const *rank_bufs, const bcast_plan_t *plan, void *cuda
     // (native, doubling) a segment is re-read on the very next hop and that still fits in L2; with
     // the tuned variant's level-order hops the re-read comes up to a tree level later and no longer
     // does (measured: 11-20 % slower than the register walk), so the tuned variant stays with registers.
-    if (mode == BCAST_EXEC_AUTO)
-        mode = ds->bandwidth_regime && p.variant != BCAST_TUNED ? BCAST_EXEC_WALK_BULK : BCAST_EXEC_WALK;
+    // It also needs at least two rounds of its own to pay: below that (about 58 MB on 148 SMs) the
+    // register walk is as fast or faster (16 MiB messages: 11 % faster).
+    if (mode == BCAST_EXEC_AUTO) {
+        const bool bulk_pays = ds->n_bulk >= 2ll * ds->bulk_grid * kBulkWorkers;
+        mode = bulk_pays && p.variant != BCAST_TUNED ? BCAST_EXEC_WALK_BULK : BCAST_EXEC_WALK;
+    }
     switch (mode) {
     case BCAST_EXEC_WALK_BULK:
         return launch_walk_bulk(p, *ds, rank_bufs, st);
