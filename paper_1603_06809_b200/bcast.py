@@ -199,7 +199,7 @@ def bcast_exec(rank_bufs, plan: Plan, stream=None) -> None:
     _check(_lib.bcast_exec(_ptr_array(rank_bufs, "rank_bufs"), plan.handle, _stream_ptr(stream)), "bcast_exec")
 
 
-def bcast_exec_mode(rank_bufs, plan: Plan, stream=None, mode: int = BCAST_EXEC_WALK) -> None:
+def bcast_exec_mode(rank_bufs, plan: Plan, stream=None, mode: int = BCAST_EXEC_AUTO) -> None:
     if len(rank_bufs) != bcast_plan_num_ranks(plan):
         raise BcastError(BCAST_ERR_INVAL, "bcast_exec_mode (len(rank_bufs) != P)")
     _check(_lib.bcast_exec_mode(_ptr_array(rank_bufs, "rank_bufs"), plan.handle, _stream_ptr(stream), mode),
@@ -245,7 +245,7 @@ def bcast_exec_status(plan: Plan) -> None:
     _check(_lib.bcast_exec_status(plan.handle), "bcast_exec_status")
 
 
-def bcast_exec_num_launches(plan: Plan, mode: int = BCAST_EXEC_WALK) -> int:
+def bcast_exec_num_launches(plan: Plan, mode: int = BCAST_EXEC_AUTO) -> int:
     return _lib.bcast_exec_num_launches(plan.handle, mode)
 
 

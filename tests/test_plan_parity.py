@@ -56,6 +56,16 @@ def test_library_exports_every_declared_symbol():
         assert hasattr(lib, name), name
 
 
+def test_binding_constants_match_header():
+    header = open(os.path.join(ROOT, "include", "bcast.h")).read()
+    pairs = dict(re.findall(r"\b(BCAST_[A-Z_]+)\s*=\s*(-?\d+)", header))
+    assert len(pairs) >= 18
+    for name, value in pairs.items():
+        assert getattr(B, name) == int(value), name
+    assert B.BCAST_MAX_RANKS == int(re.search(r"#define BCAST_MAX_RANKS (\d+)", header).group(1))
+    assert B.BCAST_STATIC_SCRATCH_BYTES == 2 << 20 and "#define BCAST_STATIC_SCRATCH_BYTES (2u << 20)" in header
+
+
 def test_xfer_layout_matches_header():
     assert B.XFER_DTYPE.itemsize == 48
     assert [B.XFER_DTYPE.fields[f][1] for f in FIELDS] == [0, 4, 8, 12, 16, 20, 24, 32, 40]
