@@ -237,3 +237,17 @@ def test_walk_order_reads_follow_writes_closely():
                 worst_plan = max(worst_plan, worst)
     assert worst_walk <= 2 * (L + 1)
     assert worst_plan > P // 2
+
+
+def test_plan_equals_oracle_random_shapes(oracle):
+    """Randomly drawn (P, root, nbytes, variant): planner and oracle agree on everything."""
+    from hypothesis import given, settings, strategies as st
+
+    @settings(max_examples=150, deadline=None, derandomize=True)
+    @given(st.integers(1, 200), st.data())
+    def check(P, data):
+        root = data.draw(st.integers(0, P - 1))
+        n = data.draw(st.one_of(st.integers(0, 4 * P + 3), st.integers(0, 1 << 22)))
+        variants = [B.BCAST_NATIVE, B.BCAST_TUNED] + ([B.BCAST_DOUBLING] if P & (P - 1) == 0 else [])
+        assert_plan_equals_oracle(oracle, P, root, n, data.draw(st.sampled_from(variants)))
+    check()
