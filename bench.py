@@ -257,6 +257,7 @@ def run_ours(args):
                 bufs[k].fill_(W.poison_byte(k))
         total_ms, per, clocks = timed(plan, args.steps, args.warmup, sample_clocks=(name == "tuned" and not args.no_clocks))
         check(name)
+        B.bcast_exec_status(plan)               # raises if a kernel gave up on one of its bounded waits
         moved = B.bcast_plan_total_bytes(plan)
         launches = B.bcast_exec_num_launches(plan, mode)
         ms_step = total_ms / args.steps
