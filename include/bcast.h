@@ -28,6 +28,10 @@
  *     tables a plan caches are only read), except in BCAST_EXEC_GRAPH mode, whose captured graph
  *     is bound to one set of buffers at a time.  The first execution of a plan (which builds those
  *     tables) must not race with another call on the same plan.
+ *   - Three environment variables override the launch shapes the library would choose, for
+ *     experiments only; they are read when a plan is executed for the first time:
+ *     BCAST_WALK_WORDS (1, 2, 4 or 8 sixteen-byte words per lane of the register walk),
+ *     BCAST_WALK_BLOCKS_PER_SM, BCAST_BULK_BLOCKS_PER_SM.
  *   - The library keeps no other global state.  There is no CPU fallback: without a CUDA device
  *     the bcast_exec* calls fail with BCAST_ERR_CUDA.
  */
