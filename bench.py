@@ -279,6 +279,9 @@ def run_ours(args):
         "algorithmic_bytes_per_launch": alg_bytes_per_launch,
         "launch_ms": round(launch_ms, 5),
         "frac_of_nominal_8TBps": round(achieved / NOMINAL_HBM_GBS, 4),
+        # the same launch counted in the DRAM bytes ncu saw (null while `traffic` is null)
+        "dram_achieved": None if traffic is None else round(traffic / (launch_ms * 1e-3) / 1e9, 1),
+        "dram_frac": None if traffic is None else round(traffic / (launch_ms * 1e-3) / 1e9 / peak, 4),
         "note": "algorithmic bytes = read + write of every scheduled byte; the read of a hop hits in L2 on what "
                 "an earlier hop stored microseconds before, so DRAM sees about half of this (every rank "
                 "buffer written once, the root's message read once): frac > 1 is expected",
