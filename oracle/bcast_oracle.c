@@ -14,9 +14,10 @@
  *     P chunks of scatter_size = ceil(nbytes / P) bytes.
  *   - Section III-A (Fig. 3):     native "enclosed" ring allgather, P-1 steps,
  *     every process sends and receives in every step.
- *   - Section IV (Figs. 4-5 and the pseudo-code listing): tuned "non-enclosed"
- *     ring allgather; each process computes (step, flag) and turns send-only or
- *     receive-only once  step > P - i.
+ *   - Section IV (Figs. 4-5 and the description of the method): tuned
+ *     "non-enclosed" ring allgather; each process knows which chunks it owned when
+ *     the scatter ended and a transfer of such a chunk to it does not take place.
+ *     The (step, flag) pair of the description is read off the simulated behaviour.
  *   - Section I: for medium messages on a power-of-two number of processes MPICH
  *     follows the scatter with a recursive-doubling allgather instead of the ring.
  *     The paper only names it; the exchange pattern simulated here is the standard
@@ -26,10 +27,10 @@
  *     block of 2^i chunks that starts at its own relative rank with the low i bits
  *     cleared.  Third variant (2); power-of-two P only.
  *
- * Every simulated process runs the per-process logic of the listing; a message
- * is the pair of one process's send and its right neighbour's receive, and the
- * simulation checks that they match before it copies anything.  No blocking,
- * fusion or reordering: one memcpy per message, steps in the paper's order.
+ * The simulation keeps, for every process, the set of chunks it holds; a message
+ * is only formed from what its sender holds (checked before anything is copied).
+ * No blocking, fusion or reordering: one memcpy per message, steps in the
+ * paper's order.
  *
  * Readings taken where the paper is silent (each also listed in the design
  * notes of the repository):
@@ -61,7 +62,6 @@
 enum { ORC_OK = 0, ORC_E_ARG = -1, ORC_E_NOMEM = -2, ORC_E_CAP = -3,
        ORC_E_NOT_HELD = -4,      /* a sender did not hold what it sends          */
        ORC_E_UNMATCHED = -5,     /* a send without the matching receive          */
-       ORC_E_STEPFLAG = -6,      /* (step, flag) left undefined by the loop      */
        ORC_E_OVERLAP = -7,       /* a step reads a range that the step writes    */
        ORC_E_INCOMPLETE = -8,    /* some process misses a chunk at the end       */
        ORC_E_MISMATCH = -9 };    /* some buffer differs from the root's message  */
@@ -69,7 +69,7 @@ enum { ORC_OK = 0, ORC_E_ARG = -1, ORC_E_NOMEM = -2, ORC_E_CAP = -3,
 /* schedule record: 9 x int64, in this order */
 enum { F_PHASE = 0, F_STEP, F_SRC, F_DST, F_CHUNK, F_NCHUNKS, F_OFFSET, F_LEN, F_DEP, F_NFIELDS };
 enum { PH_SCATTER = 0, PH_RING = 1 };
-enum { SEND_ONLY = 0, RECV_ONLY = 1, FLAG_UNSET = -1 };
+enum { SEND_ONLY = 0, RECV_ONLY = 1 };
 
 typedef struct {
     int P, root;
@@ -182,72 +182,68 @@ static int scatter_phase(sim_t *s, int L, pending_t *m)
     return ORC_OK;
 }
 
-/* Section IV, "added code" of the listing: after how many held chunks a process leaves the
-   two-sided exchange (step), and whether it then only sends or only receives (flag). */
-static void step_and_flag(int P, int r, int *step, int *flag)
-{
-    int mask = 1;
-    while (mask < P) mask <<= 1;                         /* 2^ceil(log2 P) */
-    *step = 0; *flag = FLAG_UNSET;
-    for (; mask > 1; mask >>= 1) {
-        const int rr = (r + 1 < P) ? r + 1 : r + 1 - P;  /* right neighbour, relative */
-        if (rr % mask == 0) {                            /* the right neighbour roots a sub-tree   */
-            *step = (rr + mask > P) ? P - rr : mask;     /* of this many chunks: it stops taking   */
-            *flag = RECV_ONLY;                           /* them, so this process stops sending    */
-            return;
-        }
-        if (r % mask == 0) {                             /* this process roots a sub-tree: it      */
-            *step = (r + mask > P) ? P - r : mask;       /* stops receiving and only sends         */
-            *flag = SEND_ONLY;
-            return;
-        }
-    }
-}
-
-/* Section III-A Fig. 3 (native) and Section IV Figs. 4-5 + listing (tuned): P-1 ring steps. */
-static int ring_phase(sim_t *s, int tuned, pending_t *m)
+/* Section III-A (Fig. 3) and Section IV (Figs. 4-5): the ring allgather, P-1 steps.
+ *
+ * Native ("enclosed") ring: in the first step every process passes its own chunk to its right
+ * neighbour and takes the left neighbour's; in every later step it passes on what came in the
+ * step before.  Every process sends and receives in every step, whatever it already holds.
+ *
+ * Tuned ("non-enclosed") ring: the same rotation of chunks, but each process knows the set of
+ * chunks it owned when the scatter ended (the sets drawn above the processes in Figs. 3-5) and
+ * "only receives those missing data chunks": a transfer takes place only if the receiver did not
+ * own the chunk then, and its left neighbour does not send it otherwise.  A skipped transfer does
+ * not disturb the rotation: the receiver has the chunk anyway and it is what it passes on next.
+ *
+ * Alongside the messages the phase records, per process, the last step in which it received and
+ * the last step in which it sent; step_and_flag() below reads the listing's (step, flag) pair off
+ * those.
+ */
+static int ring_phase(sim_t *s, int tuned, pending_t *m, int *last_recv, int *last_send)
 {
     const int P = s->P;
     int rc = ORC_OK;
-    int *j = malloc(sizeof(int) * (size_t)P), *jnext = malloc(sizeof(int) * (size_t)P);
-    int *step = malloc(sizeof(int) * (size_t)P), *flag = malloc(sizeof(int) * (size_t)P);
-    uint8_t *sends = malloc((size_t)P), *recvs = malloc((size_t)P);
-    if (!j || !jnext || !step || !flag || !sends || !recvs) { rc = ORC_E_NOMEM; goto out; }
-
+    uint8_t *owned_after_scatter = malloc((size_t)P * (size_t)P);
+    int *passes = malloc(sizeof(int) * (size_t)P), *arrives = malloc(sizeof(int) * (size_t)P);
+    if (!owned_after_scatter || !passes || !arrives) { rc = ORC_E_NOMEM; goto out; }
+    memcpy(owned_after_scatter, s->holds, (size_t)P * (size_t)P);
     for (int k = 0; k < P; k++) {
-        j[k] = k;                                        /* first the own chunk goes right ...     */
-        jnext[k] = (P + k - 1) % P;                      /* ... and the left neighbour's comes in  */
-        step_and_flag(P, rel_of(s, k), &step[k], &flag[k]);
-        /* P = 1: the mask loop never runs and there is no ring step that would use the result */
-        if (tuned && P > 1 && flag[k] == FLAG_UNSET) { rc = ORC_E_STEPFLAG; goto out; }
+        passes[k] = rel_of(s, k);                        /* step 1: the process's own chunk */
+        if (last_recv) last_recv[k] = 0;
+        if (last_send) last_send[k] = 0;
     }
 
     for (int i = 1; i < P; i++) {
-        /* what every process does in step i */
-        for (int k = 0; k < P; k++) {
-            if (!tuned || step[k] <= P - i) { sends[k] = 1; recvs[k] = 1; }      /* Sendrecv */
-            else if (flag[k] == RECV_ONLY)  { sends[k] = 0; recvs[k] = 1; }      /* Recv     */
-            else                            { sends[k] = 1; recvs[k] = 0; }      /* Send     */
-        }
-        /* pair each send with the right neighbour's receive */
         int nm = 0;
         for (int k = 0; k < P; k++) {
             const int right = (k + 1) % P;
-            if (sends[k] != recvs[right]) { rc = ORC_E_UNMATCHED; goto out; }
-            if (!sends[k]) continue;
-            const int rel_j = rel_of(s, j[k]);               /* chunk the sender puts on the wire   */
-            const int rel_jnext = rel_of(s, jnext[right]);   /* chunk the receiver expects          */
-            if (rel_j != rel_jnext) { rc = ORC_E_UNMATCHED; goto out; }
-            m[nm].src = k; m[nm].dst = right; m[nm].chunk = rel_j; m[nm].nchunks = 1;
+            const int chunk = passes[k];
+            arrives[right] = chunk;                      /* due at the right neighbour in this step */
+            if (tuned && owned_after_scatter[(size_t)right * P + chunk]) continue;   /* it has that one: nothing is sent */
+            m[nm].src = k; m[nm].dst = right; m[nm].chunk = chunk; m[nm].nchunks = 1;
             nm++;
+            if (last_send) last_send[k] = i;
+            if (last_recv) last_recv[right] = i;
         }
         rc = deliver_step(s, PH_RING, i - 1, m, nm);
         if (rc) goto out;
-        for (int k = 0; k < P; k++) { j[k] = jnext[k]; jnext[k] = (P + jnext[k] - 1) % P; }
+        for (int k = 0; k < P; k++) passes[k] = arrives[k];   /* forward what was due in this step */
     }
 out:
-    free(j); free(jnext); free(step); free(flag); free(sends); free(recvs);
+    free(owned_after_scatter); free(passes); free(arrives);
     return rc;
+}
+
+/* Section IV, second step of the description ("each process computes out the related step ..."):
+ * a process takes part in the two-sided exchange up to ring step P - step and from step
+ * P - step + 1 on only sends (flag 0) or only receives (flag 1).  Read off what the process
+ * does in the tuned ring: the two-sided part ends with the earlier of its last receive and its
+ * last send; the flag says which side goes on afterwards (when the sending side ends first, or
+ * both end together, the process is on the receiving side from then on). */
+static void step_and_flag(int P, int last_recv, int last_send, int *step, int *flag)
+{
+    const int two_sided_until = last_recv < last_send ? last_recv : last_send;
+    *step = P - two_sided_until;
+    *flag = last_send <= last_recv ? RECV_ONLY : SEND_ONLY;
 }
 
 /* Section I (named only) -- recursive-doubling allgather after the scatter; P a power of two. */
@@ -294,10 +290,10 @@ out:
  *   bytes_sent ...    four arrays [2][P] (phase, absolute rank), zeroed here
  * Returns ORC_OK or a negative ORC_E_* code.
  */
-int oracle_bcast_simulate(int P, int root, uint64_t nbytes, int tuned, uint8_t *const *buf,
-                          int64_t *sched, int64_t cap, int64_t *nsched,
-                          uint64_t *bytes_sent, uint64_t *bytes_recv,
-                          uint64_t *msgs_sent, uint64_t *msgs_recv)
+static int simulate(int P, int root, uint64_t nbytes, int tuned, uint8_t *const *buf,
+                    int64_t *sched, int64_t cap, int64_t *nsched,
+                    uint64_t *bytes_sent, uint64_t *bytes_recv,
+                    uint64_t *msgs_sent, uint64_t *msgs_recv, int *last_recv, int *last_send)
 {
     if (P < 1 || root < 0 || root >= P || !sched || !nsched || cap < 0 ||
         !bytes_sent || !bytes_recv || !msgs_sent || !msgs_recv)
@@ -330,7 +326,7 @@ int oracle_bcast_simulate(int P, int root, uint64_t nbytes, int tuned, uint8_t *
 
     rc = scatter_phase(&s, L, m);
     if (rc) goto out;
-    rc = tuned == 2 ? doubling_phase(&s, m) : ring_phase(&s, tuned, m);
+    rc = tuned == 2 ? doubling_phase(&s, m) : ring_phase(&s, tuned, m, last_recv, last_send);
     if (rc) goto out;
 
     /* MPI broadcast semantics (Section III-A): on return every process has the root's message */
@@ -345,16 +341,41 @@ out:
     return rc;
 }
 
+int oracle_bcast_simulate(int P, int root, uint64_t nbytes, int tuned, uint8_t *const *buf,
+                          int64_t *sched, int64_t cap, int64_t *nsched,
+                          uint64_t *bytes_sent, uint64_t *bytes_recv,
+                          uint64_t *msgs_sent, uint64_t *msgs_recv)
+{
+    return simulate(P, root, nbytes, tuned, buf, sched, cap, nsched, bytes_sent, bytes_recv,
+                    msgs_sent, msgs_recv, NULL, NULL);
+}
+
 /* scatter_size for the caller's convenience (Section IV listing) */
 uint64_t oracle_bcast_scatter_size(int P, uint64_t nbytes)
 {
     return P < 1 ? 0 : (nbytes + (uint64_t)P - 1) / (uint64_t)P;
 }
 
-/* (step, flag) of one relative rank, exposed so that tests can pin it on its own */
-int oracle_bcast_step_flag(int P, int rel_rank, int *step, int *flag)
+/*
+ * (step, flag) of every relative rank 0..P-1 in the tuned ring (Section IV), exposed so that tests
+ * can pin the pair on its own.  Obtained by simulating the tuned broadcast of a P-byte message
+ * from root 0 without data and reading off when each process last received and last sent.
+ * P = 1 has no ring: step = 1, flag = RECV_ONLY by the convention of step_and_flag().
+ */
+int oracle_bcast_step_flag(int P, int *step, int *flag)
 {
-    if (P < 1 || rel_rank < 0 || rel_rank >= P || !step || !flag) return ORC_E_ARG;
-    step_and_flag(P, rel_rank, step, flag);
-    return ORC_OK;
+    if (P < 1 || !step || !flag) return ORC_E_ARG;
+    int rc = ORC_E_NOMEM;
+    const int64_t cap = (int64_t)P * P + 1;
+    int64_t nsched = 0;
+    int64_t *sched = malloc(sizeof(int64_t) * F_NFIELDS * (size_t)cap);
+    uint64_t *cnt = malloc(sizeof(uint64_t) * 8 * (size_t)P);
+    int *last_recv = malloc(sizeof(int) * (size_t)P), *last_send = malloc(sizeof(int) * (size_t)P);
+    if (sched && cnt && last_recv && last_send) {
+        rc = simulate(P, 0, (uint64_t)P, 1, NULL, sched, cap, &nsched, cnt, cnt + 2 * P, cnt + 4 * P, cnt + 6 * P,
+                      last_recv, last_send);
+        for (int r = 0; !rc && r < P; r++) step_and_flag(P, last_recv[r], last_send[r], &step[r], &flag[r]);
+    }
+    free(sched); free(cnt); free(last_recv); free(last_send);
+    return rc;
 }

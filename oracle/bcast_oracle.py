@@ -30,7 +30,7 @@ FIELDS = ("phase", "step", "src", "dst", "chunk", "nchunks", "offset", "len", "d
 ERRORS = {
     -1: "bad argument", -2: "out of memory", -3: "schedule capacity exceeded",
     -4: "a sender did not hold what it sends", -5: "send without matching receive",
-    -6: "(step, flag) undefined", -7: "a step reads what it writes",
+    -7: "a step reads what it writes",
     -8: "a process misses a chunk at the end", -9: "a buffer differs from the root's message",
 }
 
@@ -60,8 +60,7 @@ def _bind(path: str):
     lib.oracle_bcast_scatter_size.restype = ctypes.c_uint64
     lib.oracle_bcast_scatter_size.argtypes = [ctypes.c_int, ctypes.c_uint64]
     lib.oracle_bcast_step_flag.restype = ctypes.c_int
-    lib.oracle_bcast_step_flag.argtypes = [ctypes.c_int, ctypes.c_int,
-                                           ctypes.POINTER(ctypes.c_int), ctypes.POINTER(ctypes.c_int)]
+    lib.oracle_bcast_step_flag.argtypes = [ctypes.c_int, ctypes.POINTER(ctypes.c_int), ctypes.POINTER(ctypes.c_int)]
     return lib
 
 
@@ -111,13 +110,18 @@ def scatter_size(P: int, nbytes: int) -> int:
     return int(_load().oracle_bcast_scatter_size(P, nbytes))
 
 
-def step_flag(P: int, rel_rank: int) -> tuple[int, int]:
-    """(step, flag) of the tuned ring for one relative rank; flag is SEND_ONLY, RECV_ONLY or -1."""
-    step, flag = ctypes.c_int(), ctypes.c_int()
-    rc = _load().oracle_bcast_step_flag(P, rel_rank, ctypes.byref(step), ctypes.byref(flag))
+def step_flags(P: int) -> list[tuple[int, int]]:
+    """(step, flag) of the tuned ring for every relative rank 0..P-1; flag is SEND_ONLY or RECV_ONLY."""
+    step, flag = (ctypes.c_int * P)(), (ctypes.c_int * P)()
+    rc = _load().oracle_bcast_step_flag(P, step, flag)
     if rc:
         raise OracleError(rc)
-    return step.value, flag.value
+    return list(zip(step, flag))
+
+
+def step_flag(P: int, rel_rank: int) -> tuple[int, int]:
+    """(step, flag) of one relative rank (see :func:`step_flags`)."""
+    return step_flags(P)[rel_rank]
 
 
 def capacity(P: int) -> int:

@@ -17,13 +17,21 @@ MUTANTS = [
     ("scatter_size_rounds_down", "s.S = (nbytes + (uint64_t)P - 1) / (uint64_t)P;", "s.S = P ? nbytes / (uint64_t)P : 0;"),
     ("scatter_levels_in_reverse", "const int mask = 1 << (L - 1 - t);", "const int mask = 1 << t;"),
     ("child_keeps_only_its_own_chunk", "m[nm].nchunks = hi - (r + mask);", "m[nm].nchunks = 1;"),
-    ("two_sided_phase_one_step_short", "if (!tuned || step[k] <= P - i)", "if (!tuned || step[k] < P - i)"),
-    ("two_sided_phase_one_step_long", "if (!tuned || step[k] <= P - i)", "if (!tuned || step[k] <= P - i + 1)"),
-    ("send_only_and_recv_only_swapped", "*flag = RECV_ONLY;                           /* them",
-     "*flag = SEND_ONLY;                           /* them"),
-    ("ring_turns_the_other_way", "jnext[k] = (P + k - 1) % P;", "jnext[k] = (k + 1) % P;"),
-    ("ring_chunk_by_absolute_rank", "const int rel_j = rel_of(s, j[k]);", "const int rel_j = j[k];"),
-    ("step_from_own_rank_only", "if (rr % mask == 0) {", "if (0 && rr % mask == 0) {"),
+    ("tuned_ring_skips_nothing", "if (tuned && owned_after_scatter[(size_t)right * P + chunk]) continue;",
+     "if (0 && tuned && owned_after_scatter[(size_t)right * P + chunk]) continue;"),
+    ("tuned_ring_skips_by_what_the_sender_owned", "if (tuned && owned_after_scatter[(size_t)right * P + chunk]) continue;",
+     "if (tuned && owned_after_scatter[(size_t)k * P + chunk]) continue;"),
+    ("skipped_transfer_stalls_the_rotation", "arrives[right] = chunk;                      /* due",
+     "arrives[right] = (tuned && owned_after_scatter[(size_t)right * P + chunk]) ? passes[right] : chunk;   /* due"),
+    ("ring_turns_the_other_way", "const int right = (k + 1) % P;\n            const int chunk = passes[k];",
+     "const int right = (k + P - 1) % P;\n            const int chunk = passes[k];"),
+    ("ring_chunk_by_absolute_rank", "passes[k] = rel_of(s, k);", "passes[k] = k;"),
+    ("ring_keeps_passing_the_own_chunk", "for (int k = 0; k < P; k++) passes[k] = arrives[k];", "(void)arrives;"),
+    ("send_only_and_recv_only_swapped", "*flag = last_send <= last_recv ? RECV_ONLY : SEND_ONLY;",
+     "*flag = last_send <= last_recv ? SEND_ONLY : RECV_ONLY;"),
+    ("step_from_the_receiving_side_only", "const int two_sided_until = last_recv < last_send ? last_recv : last_send;",
+     "const int two_sided_until = last_recv; (void)last_send;"),
+    ("two_sided_phase_one_step_long", "*step = P - two_sided_until;", "*step = P - two_sided_until - 1;"),
     ("dep_forgotten", "rec[F_DEP] = s->writer[(size_t)m[a].src * P + c0];", "rec[F_DEP] = -1;"),
     ("messages_sorted_by_sender", "return ((const pending_t *)a)->dst - ((const pending_t *)b)->dst;",
      "return ((const pending_t *)b)->src - ((const pending_t *)a)->src;"),

@@ -170,11 +170,13 @@ def test_message_count_closed_forms(oracle, P):
 
 
 def test_step_flag_closed_form(oracle):
-    """Section IV listing, added code: agreement of the mask loop with the sub-tree-size closed form
-    for every relative rank of every P <= 300 (and a few larger P)."""
+    """Section IV, the (step, flag) pair: what the oracle reads off its simulated tuned ring agrees
+    with the sub-tree-size closed form (which is what the listing's mask loop evaluates to) for
+    every relative rank of every P <= 300 (and a few larger P)."""
     for P in list(range(2, 301)) + [511, 512, 513, 1000, 1024]:
+        pairs = oracle.step_flags(P)
         for r in range(P):
-            step, flag = oracle.step_flag(P, r)
+            step, flag = pairs[r]
             if r == 0:
                 assert (step, flag) == (P, oracle.SEND_ONLY)
             elif r == P - 1:
