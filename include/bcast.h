@@ -247,6 +247,52 @@ int bcast_exec_static(void *const *rank_bufs, const bcast_plan_t *plan, void *cu
 int64_t bcast_plan_walk_order(const bcast_plan_t *plan, int chunk, int mode, int64_t *out, int64_t cap);
 
 /*
+ * bcast_plan_walk_pairing -- how the WALK executors carry the messages of two neighbouring chunks
+ * through a segment that holds the boundary between them.  Host only; needs no GPU.
+ * Chunks c and c+1 meet inside one 32-byte sector of every rank buffer unless scatter_size is a
+ * multiple of 32 (Section IV listing: scatter_size = ceil(nbytes / P), so usually it is not).  One
+ * warp takes the whole segment and walks a merged list of slots; a slot holds a message of chunk c,
+ * a message of chunk c+1, or one of each.  Inside each chunk the messages keep plan order (so every
+ * message still comes after the one named by its `dep`); a slot holds two messages preferably when
+ * both write the same rank, because then the sector around the boundary is written in one piece.
+ *   chunk   lower chunk c of the boundary, 0..P-2
+ *   out     HOST array of 2*cap entries (may be NULL if cap = 0): for slot i, out[2i] is the index
+ *           (into bcast_plan_xfers()) of the message of chunk c and out[2i+1] that of chunk c+1,
+ *           -1 where the slot has none
+ * Returns the number of slots (also when it exceeds cap), 0 if either chunk is empty, or a
+ * negative BCAST_ERR_* code.
+ */
+int64_t bcast_plan_walk_pairing(const bcast_plan_t *plan, int chunk, int64_t *out, int64_t cap);
+
+/*
+ * bcast_plan_walk_slices -- the units of work of the WALK executor for segments of words x 512
+ * bytes.  Host only; needs no GPU.
+ *   words   16-byte words per lane, 1..8
+ *   out     HOST array of 3*cap entries (may be NULL if cap = 0): per slice its segment index, its
+ *           kind (0: the whole segment, inside one chunk; 1: the bytes of one chunk in a segment
+ *           that the chunk does not fill; 2: a whole segment that holds one chunk boundary, see
+ *           bcast_plan_walk_pairing) and its (lower) chunk
+ * The slices of a plan cover every byte of every non-empty chunk exactly once.  Returns their
+ * number (also when it exceeds cap) or a negative BCAST_ERR_* code.
+ */
+int64_t bcast_plan_walk_slices(const bcast_plan_t *plan, int words, int64_t *out, int64_t cap);
+
+/*
+ * bcast_exec_traced -- bcast_exec_mode that also counts, on the device, the bytes it copies for
+ * every message of the plan (Sections III-A and IV count messages and their bytes per process;
+ * this is the executor's own account of them, as opposed to the planner's).
+ *   device_msg_bytes   DEVICE array of bcast_plan_num_xfers() 64-bit counters, zeroed by the
+ *                      caller; the kernels add to counter i the bytes they store for message i.
+ *                      When the enqueued work has completed, counter i equals xfers[i].len if and
+ *                      only if message i was performed in full exactly once.
+ *   mode               any mode but BCAST_EXEC_GRAPH
+ * Slower than bcast_exec_mode (one atomic per warp and hop); meant for tests and audits.
+ * Errors: as bcast_exec_mode, plus BCAST_ERR_INVAL for a NULL counter array or BCAST_EXEC_GRAPH.
+ */
+int bcast_exec_traced(void *const *rank_bufs, const bcast_plan_t *plan, void *cuda_stream, int mode,
+                      uint64_t *device_msg_bytes);
+
+/*
  * bcast_exec_status -- did a kernel of this plan give up on a bounded wait?
  * The bulk-copy kernel (BCAST_EXEC_WALK_BULK) polls an mbarrier for the arrival of every load; the
  * number of polls is limited, so that a copy that never completes ends the kernel instead of

@@ -37,7 +37,8 @@ SYMBOLS = (
     "bcast_plan", "bcast_plan_free", "bcast_plan_num_ranks", "bcast_plan_root", "bcast_plan_variant",
     "bcast_plan_nbytes", "bcast_plan_scatter_size", "bcast_plan_num_xfers", "bcast_plan_num_steps",
     "bcast_plan_xfers", "bcast_plan_step_begin", "bcast_plan_bytes_sent", "bcast_plan_bytes_recv",
-    "bcast_plan_msgs_sent", "bcast_plan_msgs_recv", "bcast_plan_total_bytes", "bcast_plan_walk_order", "bcast_exec",
+    "bcast_plan_msgs_sent", "bcast_plan_msgs_recv", "bcast_plan_total_bytes", "bcast_plan_walk_order",
+    "bcast_plan_walk_pairing", "bcast_plan_walk_slices", "bcast_exec_traced", "bcast_exec",
     "bcast_exec_mode", "bcast_exec_host", "bcast_exec_static", "bcast_exec_status", "bcast_exec_num_launches", "bcast_strerror",
     "bcast_last_cuda_error",
 )
@@ -55,6 +56,9 @@ _sig = {
     "bcast_plan_msgs_sent": (_vp, [_vp, _i]), "bcast_plan_msgs_recv": (_vp, [_vp, _i]),
     "bcast_plan_total_bytes": (_u64, [_vp]),
     "bcast_plan_walk_order": (_i64, [_vp, _i, _i, ctypes.POINTER(ctypes.c_int64), _i64]),
+    "bcast_plan_walk_pairing": (_i64, [_vp, _i, ctypes.POINTER(ctypes.c_int64), _i64]),
+    "bcast_plan_walk_slices": (_i64, [_vp, _i, ctypes.POINTER(ctypes.c_int64), _i64]),
+    "bcast_exec_traced": (_i, [_vpp, _vp, _vp, _i, _vp]),
     "bcast_exec": (_i, [_vpp, _vp, _vp]),
     "bcast_exec_mode": (_i, [_vpp, _vp, _vp, _i]),
     "bcast_exec_host": (_i, [_vpp, _vp, _vp, _i, _vp, _vpp]),
@@ -172,6 +176,29 @@ def bcast_plan_walk_order(plan: Plan, chunk: int, mode: int = BCAST_EXEC_WALK) -
     return out
 
 
+def _fill_i64(fn, plan: Plan, arg: int, width: int, where: str) -> np.ndarray:
+    """Two-call protocol of the list-returning entry points: size first, then the entries."""
+    n = fn(plan.handle, arg, None, 0)
+    if n < 0:
+        raise BcastError(int(n), where)
+    out = np.zeros((int(n), width), dtype=np.int64)
+    if n:
+        got = fn(plan.handle, arg, out.ctypes.data_as(ctypes.POINTER(ctypes.c_int64)), int(n))
+        assert got == n
+    return out
+
+
+def bcast_plan_walk_pairing(plan: Plan, chunk: int) -> np.ndarray:
+    """(slots, 2) array: per slot the message of chunk ``chunk`` and that of chunk ``chunk + 1``
+    (indices into the schedule, -1 where the slot has none)."""
+    return _fill_i64(_lib.bcast_plan_walk_pairing, plan, chunk, 2, "bcast_plan_walk_pairing")
+
+
+def bcast_plan_walk_slices(plan: Plan, words: int) -> np.ndarray:
+    """(slices, 3) array: segment index, kind (0 whole / 1 ragged / 2 dual), (lower) chunk."""
+    return _fill_i64(_lib.bcast_plan_walk_slices, plan, words, 3, "bcast_plan_walk_slices")
+
+
 def _ptr_array(items, what: str):
     """A C array of pointers from ints, objects with ``data_ptr()`` (torch tensors) or None."""
     vals = []
@@ -204,6 +231,16 @@ def bcast_exec_mode(rank_bufs, plan: Plan, stream=None, mode: int = BCAST_EXEC_A
         raise BcastError(BCAST_ERR_INVAL, "bcast_exec_mode (len(rank_bufs) != P)")
     _check(_lib.bcast_exec_mode(_ptr_array(rank_bufs, "rank_bufs"), plan.handle, _stream_ptr(stream), mode),
            "bcast_exec_mode")
+
+
+def bcast_exec_traced(rank_bufs, plan: Plan, stream, mode: int, device_msg_bytes) -> None:
+    """``device_msg_bytes``: device pointer (int) or CUDA tensor of ``num_xfers`` zeroed 64-bit
+    counters; the kernels add the bytes they store for every message."""
+    if len(rank_bufs) != bcast_plan_num_ranks(plan):
+        raise BcastError(BCAST_ERR_INVAL, "bcast_exec_traced (len(rank_bufs) != P)")
+    ptr = device_msg_bytes.data_ptr() if hasattr(device_msg_bytes, "data_ptr") else int(device_msg_bytes)
+    _check(_lib.bcast_exec_traced(_ptr_array(rank_bufs, "rank_bufs"), plan.handle, _stream_ptr(stream), mode,
+                                  ctypes.c_void_p(ptr)), "bcast_exec_traced")
 
 
 def bcast_exec_host(rank_bufs, plan: Plan, stream, mode: int, host_message, host_out=None) -> None:

@@ -184,6 +184,7 @@ void bcast_plan_free(bcast_plan_t *plan)
 {
     if (!plan) return;
     bcast_device_state_free(plan->dev);
+    bcast_static_image_free(plan->static_img);
     delete plan;
 }
 

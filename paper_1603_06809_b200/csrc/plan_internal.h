@@ -6,6 +6,7 @@
 #include "bcast.h"
 
 struct bcast_device_state;   // defined in exec.cu; owns the device tables cached by a plan
+struct bcast_static_image;   // defined in exec.cu; host image of the tables bcast_exec_static uses
 
 struct bcast_plan {
     int P = 0, root = 0, variant = 0;
@@ -16,7 +17,10 @@ struct bcast_plan {
     std::vector<uint64_t> bytes_sent[2], bytes_recv[2], msgs_sent[2], msgs_recv[2];   // [phase][rank]
     uint64_t total_bytes = 0;
     mutable bcast_device_state *dev = nullptr;  // created by the first execution
+    mutable bcast_static_image *static_img = nullptr;   // created by the first bcast_exec_static (host memory only)
 };
 
 // exec.cu: frees the cached device tables of a plan (no-op when there are none)
 void bcast_device_state_free(bcast_device_state *dev);
+// exec.cu: frees the host image kept for bcast_exec_static (no-op when there is none)
+void bcast_static_image_free(bcast_static_image *img);
