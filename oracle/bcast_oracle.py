@@ -169,3 +169,47 @@ def simulate(P: int, root: int, nbytes: int, variant: int, message: np.ndarray |
                         schedule=sched[: nsched.value].copy(),
                         bytes_sent=cnt[0], bytes_recv=cnt[1], msgs_sent=cnt[2], msgs_recv=cnt[3],
                         bufs=bufs, seconds=dt)
+
+
+# ---- the all-cores CPU baseline: the oracle's schedule replayed by a team of threads
+_SRC_MT = os.path.join(_HERE, "bcast_oracle_mt.c")
+_LIB_MT = os.path.join(_HERE, "_build", "libbcast_oracle_mt.so")
+_lib_mt = None
+
+
+def build_mt(force: bool = False) -> str:
+    """Compile oracle/bcast_oracle_mt.c (pthreads) if missing or stale."""
+    if force or not os.path.exists(_LIB_MT) or os.path.getmtime(_LIB_MT) < os.path.getmtime(_SRC_MT):
+        os.makedirs(os.path.dirname(_LIB_MT), exist_ok=True)
+        tmp = _LIB_MT + f".{os.getpid()}.tmp"
+        subprocess.check_call(["gcc", "-O2", "-Wall", "-Wextra", "-pthread", "-shared", "-fPIC", "-o", tmp, _SRC_MT])
+        os.replace(tmp, _LIB_MT)
+    return _LIB_MT
+
+
+def replay_mt(P: int, schedule: np.ndarray, bufs: np.ndarray, nthreads: int) -> float:
+    """Perform the messages of ``schedule`` (as returned by :func:`simulate`) on ``bufs`` ((P, nbytes)
+    uint8, the root's row holding the message) with ``nthreads`` threads, step by step with a barrier
+    after every step.  Returns the wall time in seconds.  Only the benchmark's all-cores CPU baseline
+    and the test that compares its buffers with the single-threaded oracle's use this."""
+    global _lib_mt
+    if _lib_mt is None:
+        _lib_mt = ctypes.CDLL(build_mt())
+        _lib_mt.oracle_bcast_replay_mt.restype = ctypes.c_int
+        _lib_mt.oracle_bcast_replay_mt.argtypes = [
+            ctypes.c_int, ctypes.POINTER(ctypes.c_void_p), ctypes.POINTER(ctypes.c_int64), ctypes.c_int64,
+            ctypes.c_int, ctypes.POINTER(ctypes.c_double)]
+    assert bufs.dtype == np.uint8 and bufs.ndim == 2 and bufs.shape[0] == P and bufs.flags.c_contiguous
+    sched = np.ascontiguousarray(schedule, dtype=np.int64)
+    assert sched.ndim == 2 and sched.shape[1] == len(FIELDS)
+    nbytes = bufs.shape[1]
+    if len(sched):
+        assert int((sched[:, FIELDS.index("offset")] + sched[:, FIELDS.index("len")]).max()) <= nbytes
+    base = bufs.ctypes.data
+    ptrs = (ctypes.c_void_p * P)(*[base + k * nbytes for k in range(P)])
+    seconds = ctypes.c_double(0.0)
+    rc = _lib_mt.oracle_bcast_replay_mt(P, ptrs, sched.ctypes.data_as(ctypes.POINTER(ctypes.c_int64)), len(sched),
+                                        nthreads, ctypes.byref(seconds))
+    if rc:
+        raise OracleError(rc)
+    return seconds.value

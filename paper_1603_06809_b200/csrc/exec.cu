@@ -200,14 +200,14 @@ int walk_blocks_per_sm(int u, int P, int *bps)
 // in flight than needed: about 32 KB per SM (8 warps x 8 words x 512 B) saturate the memory
 // system; more concurrent slices scatter the DRAM writes further and, with level-order hops,
 // push the copies that are still to be re-read out of L2.
-//   * Message larger than that (more than 1.4 rounds of SMs x 32 KB): one block per SM, several
-//     rounds.  All slices take the same time, so a last round that only some warps take part in
-//     costs nearly a whole round: of U = 8, 7, 6, 5 the one whose last round is fullest is taken.
+//   * Message larger than that (more than 1.4 rounds of SMs x 32 KB): U = 8, one block per SM,
+//     several rounds.  (Smaller segments that would fill the last round better were measured and
+//     lose: 3.5 rounds of 4 KiB segments beat 4.0 rounds of 3.5 KiB ones by 6 %.)
 //   * Smaller: everything is in flight at once and the run time is one walk down the longest hop
 //     list at memory latency; take the smallest U whose slices fit the resident warps (the most
 //     warps, the fewest words each).
 //   * Very few ranks (P <= 4): at most three hops per slice, close to a plain copy: as many
-//     bytes in flight as the SMs hold.
+//     bytes in flight as the SMs hold (U = 4 for P <= 3, U = 2 for P = 4, all resident blocks).
 // BCAST_WALK_WORDS and BCAST_WALK_BLOCKS_PER_SM override the choice (for experiments).
 struct WalkShape {
     int u = 1, grid = 1;
@@ -224,17 +224,11 @@ int choose_walk_shape(const bcast_plan_t &p, int sm_count, WalkShape *shape)
         if ((rc = walk_blocks_per_sm(u, p.P, &resident))) return rc;
         bps = forced_bps > 0 ? std::min(forced_bps, resident) : resident;
     } else if (p.P <= 4) {
-        u = 2;
+        u = p.P <= 3 ? 4 : 2;
         if ((rc = walk_blocks_per_sm(u, p.P, &resident))) return rc;
         bps = resident;
     } else if (count_slices(p, 512ull * kMaxWords, true) * 5 > (long long)sm_count * kWarpsPerBlock * 7) {   // > 1.4 rounds
-        double best = -1.0;
-        for (int cand = kMaxWords; cand >= 5; cand--) {
-            const long long per_sm = (count_slices(p, 512ull * cand, true) + sm_count - 1) / sm_count;
-            const long long rounds = (per_sm + kWarpsPerBlock - 1) / kWarpsPerBlock;
-            const double fill = (double)per_sm / (double)(rounds * kWarpsPerBlock);
-            if (fill > best + 0.02) { best = fill; u = cand; }      // larger U wins unless a smaller one fills clearly better
-        }
+        u = kMaxWords;
         bps = 1;
     } else {
         for (int cand = 1; cand <= kMaxWords; cand++) {
@@ -275,7 +269,7 @@ int build_walk_tables(const bcast_plan_t &p, bcast_device_state &ds)
     ds.walk_u = shape.u;
     ds.walk_grid = shape.grid;
     std::vector<WalkSlice> slices;
-    make_slices(p, 512ull * ds.walk_u, true, slices);
+    make_slices(p, 512ull * ds.walk_u, env_int("BCAST_WALK_DUAL", 1) != 0, slices);
     ds.n_slices = (long long)slices.size();
     return upload(&ds.d_slices, slices);
 }

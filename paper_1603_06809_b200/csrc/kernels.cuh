@@ -88,6 +88,15 @@ __device__ __forceinline__ void st1(uint8_t *p, uint32_t v)
     asm volatile("st.global.u8 [%0], %1;" :: "l"(p), "r"(v) : "memory");
 }
 
+// Ask L2 to fetch the line that holds *p.  Used ahead of a store that will cover only part of a
+// 32-byte sector: a sector that sits in L2 partly written makes the next read of it wait for
+// DRAM, whereas a partial write into a sector that is already complete in L2 leaves it complete.
+__device__ __forceinline__ void prefetch_l2(const uint8_t *p)
+{
+    asm volatile("prefetch.global.L2 [%0];" :: "l"(p) : "memory");
+}
+constexpr int kPrefetchAhead = 6;         // hops between that request and the partial store
+
 // Warp-wide: add the bytes the lanes stored for plan message `msg` to its counter.
 __device__ __forceinline__ void trace_add(unsigned long long *trace, int msg, uint32_t lane_bytes)
 {
@@ -165,6 +174,13 @@ __device__ __forceinline__ void walk_ragged(const RankPtrs<MAXP> &bufs, uint32_t
     uint32_t e = __ldg(hp);
     const uint8_t *s = bufs.p[e & 0xffffu];
     uint8_t *d = bufs.p[e >> 16];
+    // the first and the last sector of the range may be written in part only: have them in L2 first
+    for (int h = (int)lane; h < min(nh, kPrefetchAhead); h += 32) {
+        uint8_t *dn = bufs.p[__ldg(hp + h) >> 16];
+        prefetch_l2(dn + lo);
+        prefetch_l2(dn + hi - 1);
+    }
+    uint32_t ahead = __ldg(hp + min(kPrefetchAhead, nh - 1));
     for (int h = 0; h < nh; h++) {
         uint4 v[U];
         uint32_t b = 0;
@@ -172,6 +188,11 @@ __device__ __forceinline__ void walk_ragged(const RankPtrs<MAXP> &bufs, uint32_t
         for (int u = 0; u < U; u++)
             if (ok[u]) v[u] = ld16(s + base + (uint64_t)u * 512);
         if (has_edge) b = ld1(s + eoff);
+        if (lane < 2 && h + kPrefetchAhead < nh) {
+            uint8_t *dn = bufs.p[ahead >> 16];
+            prefetch_l2(lane ? dn + hi - 1 : dn + lo);
+        }
+        ahead = __ldg(hp + min(h + 1 + kPrefetchAhead, nh - 1));   // fetched a hop early: nothing waits for it
         e = __ldg(hp + min(h + 1, nh - 1));
         const uint8_t *s_next = bufs.p[e & 0xffffu];
         uint8_t *d_next = bufs.p[e >> 16];
@@ -204,12 +225,17 @@ __device__ __forceinline__ void store_bytes(uint8_t *p, const uint4 &v, uint32_t
 
 // A whole segment that holds exactly one chunk boundary (`cut` bytes into it): the words below it
 // follow the hops of chunk c, the words above it those of chunk c+1, slot by slot of the
-// boundary's dual list.  The 16-byte word that straddles the boundary (if the boundary is not a
-// multiple of 16) belongs to one lane, which loads it from both sources; when the two hops of a
-// slot write the same rank it stores the word whole -- its low `cut % 16` bytes from the lower
-// chunk's source, the rest from the upper chunk's -- so that the 32-byte sector around the
-// boundary is written by ONE warp instruction and never sits half-written in L2.  Otherwise
-// (a slot with one hop, or two different destinations) the parts go out byte by byte.
+// boundary's dual list.
+//   * A slot whose two hops are the same (src, dst) pair -- every ring step once the lists are
+//     aligned -- moves the segment as one piece, exactly like a full slice.
+//   * Otherwise every lane takes source, destination and predicate from the side its word is on.
+//     The 16-byte word that straddles the boundary (if the boundary is not a multiple of 16)
+//     belongs to one lane, which loads it from both sources; when the two hops write the same
+//     rank it stores the word whole -- its low `cut % 16` bytes from the lower chunk's source, the
+//     rest from the upper chunk's -- in the same warp instruction as its neighbours, so that the
+//     32-byte sector around the boundary is written in one piece and never sits half-written in
+//     L2 (a read of a half-written sector has to wait for DRAM).  With one hop only, or two
+//     different destinations, the parts go out byte by byte.
 template <int U, int MAXP, bool TRACE>
 __device__ __forceinline__ void walk_dual(const RankPtrs<MAXP> &bufs, uint32_t seg, uint32_t c, const WalkDev &t,
                                           uint32_t lane)
@@ -219,10 +245,12 @@ __device__ __forceinline__ void walk_dual(const RankPtrs<MAXP> &bufs, uint32_t s
     const uint32_t cut = (uint32_t)(((uint64_t)c + 1) * t.scatter_size - seg_lo);   // 0 < cut < kSeg
     const int s0 = t.dual_begin[c];
     const int ns = t.dual_begin[c + 1] - s0;
+    if (ns <= 0) return;
     const DualSlot *sp = t.dual + s0;
     const uint64_t base = seg_lo + (uint64_t)lane * 16;
     const uint32_t k = cut & 15u;                                   // bytes of the straddling word below the boundary
-    const bool strad = k != 0 && lane == ((cut >> 4) & 31u);        // this lane owns the straddling word
+    const bool strad = k != 0 && lane == ((cut >> 4) & 31u);        // this lane owns the straddling word ...
+    const int su = (int)(cut >> 9);                                 // ... as its word number su
     const uint64_t so = seg_lo + (cut & ~15u);
     uint32_t bytes_a = 0, bytes_b = 0;
     if constexpr (TRACE) {
@@ -234,45 +262,67 @@ __device__ __forceinline__ void walk_dual(const RankPtrs<MAXP> &bufs, uint32_t s
         }
         if (strad) { bytes_a += k; bytes_b += 16u - k; }
     }
+    DualSlot e = sp[0];
+    // slots whose two hops differ store only part of the sector around the boundary: have it in L2
+    // first.  The scatter hops, where most such slots are, come first: one request per lane now;
+    // for the others the table flags the slot kDualAhead places before.
+    auto prefetch_cut = [&](int slot) {
+        const DualSlot a = sp[slot];
+        if (a.a == a.b) return;
+        if (a.a != kNoHop) prefetch_l2(bufs.p[a.a >> 16] + seg_lo + cut - 1);
+        if (a.b != kNoHop) prefetch_l2(bufs.p[a.b >> 16] + seg_lo + cut);
+    };
+    if ((int)lane < min(ns, kDualAhead)) prefetch_cut((int)lane);
     for (int h = 0; h < ns; h++) {
-        const DualSlot e = sp[h];
-        const bool ha = e.a != kNoHop, hb = e.b != kNoHop;
-        const uint8_t *sa = bufs.p[ha ? (e.a & 0xffffu) : 0u], *sb = bufs.p[hb ? (e.b & 0xffffu) : 0u];
-        uint8_t *da = bufs.p[ha ? (e.a >> 16) : 0u], *db = bufs.p[hb ? (e.b >> 16) : 0u];
-        uint4 v[U], wa, wb;
+        const DualSlot cur = e;
+        if (cur.a == cur.b) {
+            // the same hop for both chunks: the segment moves as one piece
+            const uint8_t *s = bufs.p[cur.a & kHopRankMask];
+            uint8_t *d = bufs.p[cur.a >> 16];
+            uint4 v[U];
 #pragma unroll
-        for (int u = 0; u < U; u++) {
-            const uint32_t o = lane * 16u + (uint32_t)u * 512u;
-            if (o + 16 <= cut) { if (ha) v[u] = ld16(sa + base + (uint64_t)u * 512); }
-            else if (o >= cut) { if (hb) v[u] = ld16(sb + base + (uint64_t)u * 512); }
-        }
-        if (strad) {
-            if (ha) wa = ld16(sa + so);
-            if (hb) wb = ld16(sb + so);
-        }
+            for (int u = 0; u < U; u++) v[u] = ld16(s + base + (uint64_t)u * 512);
+            e = sp[min(h + 1, ns - 1)];                  // next slot, while the loads are in flight
+            if (lane == 0 && (cur.a & kHopAheadFlag)) prefetch_cut(h + kDualAhead);
 #pragma unroll
-        for (int u = 0; u < U; u++) {
-            const uint32_t o = lane * 16u + (uint32_t)u * 512u;
-            if (o + 16 <= cut) { if (ha) st16(da + base + (uint64_t)u * 512, v[u]); }
-            else if (o >= cut) { if (hb) st16(db + base + (uint64_t)u * 512, v[u]); }
-        }
-        if (strad) {
-            if (ha && hb && da == db) {
-                uint4 m;
-                m.x = low_bytes_from(wa.x, wb.x, (int)k);
-                m.y = low_bytes_from(wa.y, wb.y, (int)k - 4);
-                m.z = low_bytes_from(wa.z, wb.z, (int)k - 8);
-                m.w = low_bytes_from(wa.w, wb.w, (int)k - 12);
-                st16(da + so, m);
-            } else {
+            for (int u = 0; u < U; u++) st16(d + base + (uint64_t)u * 512, v[u]);
+        } else {
+            const bool ha = cur.a != kNoHop, hb = cur.b != kNoHop;
+            const uint8_t *sa = bufs.p[ha ? (cur.a & kHopRankMask) : 0u], *sb = bufs.p[hb ? (cur.b & kHopRankMask) : 0u];
+            uint8_t *da = bufs.p[ha ? (cur.a >> 16) : 0u], *db = bufs.p[hb ? (cur.b >> 16) : 0u];
+            const bool whole = ha && hb && da == db;     // the straddling word can be stored in one piece
+            uint4 v[U], wa = make_uint4(0, 0, 0, 0), wb = wa;
+#pragma unroll
+            for (int u = 0; u < U; u++) {
+                const uint32_t o = lane * 16u + (uint32_t)u * 512u;
+                const bool upper = o >= cut;             // else lower, or the straddling word (loaded from the lower source here)
+                if (upper ? hb : ha) v[u] = ld16((upper ? sb : sa) + base + (uint64_t)u * 512);
+            }
+            if (strad && hb) wb = ld16(sb + so);
+            e = sp[min(h + 1, ns - 1)];
+            if (lane == 0 && ((ha ? cur.a : cur.b) & kHopAheadFlag)) prefetch_cut(h + kDualAhead);
+#pragma unroll
+            for (int u = 0; u < U; u++) {
+                const uint32_t o = lane * 16u + (uint32_t)u * 512u;
+                const bool upper = o >= cut, mine = strad && u == su;
+                if (mine) {
+                    wa = v[u];
+                    v[u].x = low_bytes_from(wa.x, wb.x, (int)k);
+                    v[u].y = low_bytes_from(wa.y, wb.y, (int)k - 4);
+                    v[u].z = low_bytes_from(wa.z, wb.z, (int)k - 8);
+                    v[u].w = low_bytes_from(wa.w, wb.w, (int)k - 12);
+                }
+                if (mine ? whole : (upper ? hb : ha)) st16((upper ? db : da) + base + (uint64_t)u * 512, v[u]);
+            }
+            if (strad && !whole) {
                 if (ha) store_bytes(da + so, wa, 0u, k);
                 if (hb) store_bytes(db + so, wb, k, 16u);
             }
         }
         if constexpr (TRACE) {
             const DualMsg m = t.dual_msg[s0 + h];
-            trace_add(t.trace, m.a, ha ? bytes_a : 0u);
-            trace_add(t.trace, m.b, hb ? bytes_b : 0u);
+            trace_add(t.trace, m.a, cur.a != kNoHop ? bytes_a : 0u);
+            trace_add(t.trace, m.b, cur.b != kNoHop ? bytes_b : 0u);
         }
     }
 }

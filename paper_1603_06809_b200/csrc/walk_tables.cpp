@@ -134,9 +134,18 @@ void make_walk_tables(const bcast_plan_t &p, WalkTables &t)
         t.dual_begin[c] = (int)t.dual.size();
         if (c + 1 >= P || per_chunk[c].empty() || per_chunk[c + 1].empty()) continue;
         pair_hops(p, per_chunk[c], per_chunk[c + 1], slots);
+        const size_t first = t.dual.size();
         for (const DualMsg &s : slots) {
             t.dual.push_back(DualSlot{s.a < 0 ? kNoHop : encode_hop(p, s.a), s.b < 0 ? kNoHop : encode_hop(p, s.b)});
             t.dual_msg.push_back(s);
+        }
+        // mark the slots that come kDualAhead before a slot with two different hops (see kHopAheadFlag)
+        for (size_t i = 0; i + kDualAhead < slots.size(); i++) {
+            const DualSlot &ahead = t.dual[first + i + kDualAhead];
+            if ((ahead.a & ~kHopAheadFlag) == (ahead.b & ~kHopAheadFlag)) continue;
+            DualSlot &now = t.dual[first + i];
+            if (now.a != kNoHop) now.a |= kHopAheadFlag;
+            if (now.b != kNoHop) now.b |= kHopAheadFlag;
         }
     }
     t.dual_begin[P] = (int)t.dual.size();

@@ -24,6 +24,11 @@ constexpr uint32_t kSliceRefMask = (1u << kSliceKindShift) - 1u;
 // A hop is src_rank | dst_rank << 16.  A slot of a dual list holds one hop of the lower chunk
 // (a) and one of the upper chunk (b), either of which may be absent.
 constexpr uint32_t kNoHop = 0xffffffffu;
+// Dual slots only: bit 15 of a hop says that the slot kDualAhead places further on holds two
+// different hops (or one), i.e. will store only part of the sector around the boundary; the warp
+// then asks L2 for that sector now.  Ranks need 10 bits, so the source rank is hop & kHopRankMask.
+constexpr uint32_t kHopAheadFlag = 0x8000u, kHopRankMask = 0x3ffu;
+constexpr int kDualAhead = 6;
 struct DualSlot {
     uint32_t a, b;
 };
