@@ -57,15 +57,15 @@ def parse_args():
 
 # DRAM bytes of one launch of the dominant kernel (tuned variant), from ncu:
 # dram__bytes_read.sum + dram__bytes_write.sum.  A figure is only valid for the kernel source it
-# was taken with, so each carries the SHA-256 of the device code in csrc/exec.cu; once that
+# was taken with, so each carries the SHA-256 of the device code (csrc/kernels.cuh); once that
 # changes, `traffic` is reported as null until the counters are taken again.
 NCU_TRAFFIC = {
     # profiles/bcast_walk_kernel_P100_64MiB_launch_list_and_dram.md
-    ("cfg4", "walk"): {"dram_bytes_per_launch": 68251904 + 6586495232,
-                       "kernel_sha256": "50efc9471b3c11348ddb50cfcdd1062cef41bb49f5885f140d967d68364c17bc"},
-    # profiles/bcast_walk_kernel_P64_16MiB_ncu_full.md (same one-pass metric pair, cfg3)
-    ("cfg3", "walk"): {"dram_bytes_per_launch": 17160448 + 999243520,
-                       "kernel_sha256": "50efc9471b3c11348ddb50cfcdd1062cef41bb49f5885f140d967d68364c17bc"},
+    ("cfg4", "walk"): {"dram_bytes_per_launch": 68683264 + 6586248704,
+                       "kernel_sha256": "d6f58d59f8b3f871f4623b6952b853624023556e5db5fe3b268416353515faae"},
+    # same file, last paragraph (same one-pass metric pair, cfg3)
+    ("cfg3", "walk"): {"dram_bytes_per_launch": 17548544 + 998966528,
+                       "kernel_sha256": "d6f58d59f8b3f871f4623b6952b853624023556e5db5fe3b268416353515faae"},
 }
 
 
@@ -144,6 +144,16 @@ class ClockSampler:
         res = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0, "power_w": None}
         if self.proc is None:
             return res
+        # nvidia-smi needs some tens of milliseconds to come up: if the timed region was shorter
+        # than that, wait (bounded) for its first samples, which are then the nearest ones
+        deadline = time.time() + 1.5
+        while time.time() < deadline:
+            try:
+                if os.path.getsize(self.path) > 200:
+                    break
+            except OSError:
+                break
+            time.sleep(0.02)
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
@@ -360,6 +370,27 @@ def run_ours(args):
                "ms_per_step": round(dt / args.e2e_steps * 1e3, 3),
                "what": "bcast_exec_host: pinned host message -> root buffer, broadcast, all P rank buffers -> pinned host"}
         del host_out, outs
+
+    # ---- context for the roofline: what plain sequential stores reach on this GPU (no loads at all).
+    # Overwrites the rank buffers, so it comes last.  torch's fill kernel on a 32-bit view: library
+    # plumbing, not part of the broadcast.
+    try:
+        flat = bufs.view(-1)[: bufs.numel() // 4 * 4].view(torch.int32)
+        for _ in range(2):
+            flat.fill_(7)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record(stream)
+        for _ in range(5):
+            flat.fill_(9)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        fill_gbs = flat.numel() * 4 * 5 / (e0.elapsed_time(e1) * 1e-3) / 1e9
+        roofline["write_only_reference"] = {
+            "GBps": round(fill_gbs, 1), "how": "torch fill_ of the rank buffers (int32 view), sequential stores, 5 passes",
+            "dram_write_rate_of_this_kernel_GBps": round((P - 1) * n / launches / (launch_ms * 1e-3) / 1e9, 1)}
+    except Exception as e:
+        roofline["write_only_reference"] = {"error": str(e)[:120]}
 
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:

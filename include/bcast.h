@@ -27,11 +27,18 @@
  *     the same plan may overlap on the GPU if they use different rank buffers (the device-side
  *     tables a plan caches are only read), except in BCAST_EXEC_GRAPH mode, whose captured graph
  *     is bound to one set of buffers at a time.  The first execution of a plan (which builds those
- *     tables) must not race with another call on the same plan.
- *   - Three environment variables override the launch shapes the library would choose, for
- *     experiments only; they are read when a plan is executed for the first time:
- *     BCAST_WALK_WORDS (1, 2, 4 or 8 sixteen-byte words per lane of the register walk),
- *     BCAST_WALK_BLOCKS_PER_SM, BCAST_BULK_BLOCKS_PER_SM.
+ *     tables) must not race with another call on the same plan; later calls on one plan may come
+ *     from several host threads (the plan's host-side caches are locked).  The rank-buffer check
+ *     is skipped for the set of pointers that passed it last, on the assumption that those
+ *     buffers are still allocated.
+ *   - Environment variables override what the library would choose, for experiments and tests
+ *     only; they are read when a plan is executed for the first time (the last one at every call):
+ *     BCAST_WALK_WORDS (1..8 sixteen-byte words per lane of the register walk, i.e. segments of
+ *     512 B .. 4 KiB), BCAST_WALK_BLOCKS_PER_SM, BCAST_BULK_BLOCKS_PER_SM, BCAST_WALK_DUAL (0: walk
+ *     a segment that holds a chunk boundary in two parts instead of with the merged list of
+ *     bcast_plan_walk_pairing), BCAST_BULK_SPIN_LIMIT (polls of the bulk-copy kernel's first wait
+ *     bound, see bcast_exec_status; 0 makes every wait report a timeout and then complete under the
+ *     second bound), BCAST_BULK_PLAN_ORDER (1: the bulk walk takes the hops in plan order).
  *   - The library keeps no other global state.  There is no CPU fallback: without a CUDA device
  *     the bcast_exec* calls fail with BCAST_ERR_CUDA.
  */
@@ -66,13 +73,14 @@ enum {
 /* How bcast_exec_mode() runs a plan.  All modes perform exactly the plan's messages. */
 enum {
     /* One launch for the whole plan.  The message is cut into segments on a fixed grid of byte
-       offsets (and at chunk boundaries); a warp takes such a slice and carries it through every
-       message of the plan that covers it (scatter hops and ring hops), re-reading it from the
-       source rank's buffer at every hop.  Messages that cover different byte ranges are
-       independent, so no waiting between warps is needed.  The hops of a slice run in an order
-       that respects every `dep` of the plan (no copy is read before the message that delivers it
-       has been performed) but is not the plan's step order where a different order keeps the
-       data in L2: see BCAST_EXEC_WALK_PLAN_ORDER. */
+       offsets; a warp takes a segment and carries it through every message of the plan that
+       covers it (scatter hops and ring hops), re-reading it from the source rank's buffer at
+       every hop.  Messages that cover different byte ranges are independent, so no waiting
+       between warps is needed.  A segment that holds the boundary between two chunks is carried
+       through both chunks' messages at once (bcast_plan_walk_pairing).  The hops of a segment
+       run in an order that respects every `dep` of the plan (no copy is read before the message
+       that delivers it has been performed) but is not the plan's step order where a different
+       order keeps the data in L2: see BCAST_EXEC_WALK_PLAN_ORDER. */
     BCAST_EXEC_WALK = 0,
     /* One launch per plan step (ceil(log2 P) + P - 1 launches) on the caller's stream; inside a
        launch the messages of that step are cut into tiles and copied in parallel. */
@@ -215,19 +223,29 @@ int bcast_exec_host(void *const *rank_bufs, const bcast_plan_t *plan, void *cuda
  *   rank_bufs, plan, cuda_stream   as for bcast_exec(); inputs and outputs are still the caller's.
  * Behaviour to know about:
  *   - Plans whose tables do not fit (roughly: 8 B per slice of the message -- slices are 512 B to
- *     4 KiB, the larger size is tried before giving up -- plus 4 B per (chunk, message) pair,
- *     about 4*P*P bytes) are refused with BCAST_ERR_CAPACITY before
- *     anything is copied or launched.  All configurations up to P = 256 ranks with messages up to
- *     512 MiB fit; P = 1024 does not.
+ *     4 KiB -- plus 4 B per (chunk, message) pair, about 4*P*P bytes, plus, when there is room, 8 B
+ *     per (chunk boundary, message) pair for the lists of bcast_plan_walk_pairing) are refused
+ *     with BCAST_ERR_CAPACITY before anything is copied or launched.  The call tries, in this
+ *     order: everything; without the boundary lists (segments that hold a chunk boundary are then
+ *     walked in two parts, which is slower for odd scatter sizes, never wrong); the largest slices.
+ *     All configurations up to P = 256 ranks with messages up to 256 MiB fit; P = 1024 does not.
  *   - The first call on a device looks up the array's device address (cudaGetSymbolAddress) and
- *     remembers it; make that first call outside any stream capture.
- *   - Every call re-writes the array (stream-ordered on cuda_stream) from host memory, so its
- *     previous contents never matter; nothing in it has to start at zero (the kernel only reads it).
+ *     remembers it.
+ *   - Never call it on a stream that is being captured into a CUDA graph: the call returns
+ *     BCAST_ERR_INVAL in that case.  (It copies the tables into the one shared array; recorded into
+ *     a graph, that copy would be replayed later from memory that may have changed.)
+ *   - Every call re-writes the array (stream-ordered on cuda_stream) from host memory that the plan
+ *     keeps, so its previous contents never matter; nothing in it has to start at zero (the kernel
+ *     only reads it).  The copy's source is ordinary pageable memory, so the call may block the
+ *     host until earlier work on cuda_stream has finished; unlike bcast_exec it is not purely
+ *     asynchronous.
  *     Because all calls share the one array, two calls whose GPU work overlaps in time (different
  *     streams, or different host threads) race on it: serialise them.
+ *   - The rank buffers are checked like in bcast_exec; the set that passed last is remembered per
+ *     device, on the assumption that those buffers stay allocated.
  *   - No cudaMalloc, cudaFree or other allocating CUDA call is made; ordinary host heap memory is
- *     used briefly to assemble the tables.
- * Errors: BCAST_ERR_INVAL as for bcast_exec, BCAST_ERR_CAPACITY, BCAST_ERR_CUDA.
+ *     used to assemble the tables (once per plan).
+ * Errors: BCAST_ERR_INVAL as for bcast_exec or for a capturing stream, BCAST_ERR_CAPACITY, BCAST_ERR_CUDA.
  */
 #define BCAST_STATIC_SCRATCH_BYTES (2u << 20)
 int bcast_exec_static(void *const *rank_bufs, const bcast_plan_t *plan, void *cuda_stream);
@@ -296,10 +314,13 @@ int bcast_exec_traced(void *const *rank_bufs, const bcast_plan_t *plan, void *cu
  * bcast_exec_status -- did a kernel of this plan give up on a bounded wait?
  * The bulk-copy kernel (BCAST_EXEC_WALK_BULK) polls an mbarrier for the arrival of every load; the
  * number of polls is limited, so that a copy that never completes ends the kernel instead of
- * hanging the GPU.  A worker whose limit runs out sets a flag in the plan's device state and stops;
- * the rank buffers are then incomplete.  Call this after the stream has been synchronised: it reads
- * the flag (a blocking 4-byte copy), clears it, and returns BCAST_ERR_TIMEOUT if it was set, else
- * BCAST_OK.  The other executors have no waits and never set it.
+ * hanging the GPU.  A worker whose first limit runs out sets a flag in the plan's device state and
+ * goes on waiting under a second, much larger limit (it must not leave while its own copy may still
+ * be landing in the block's shared memory); if the load arrives after all, the worker carries on
+ * and the rank buffers end up complete; if the second limit runs out too, the worker stops and the
+ * rank buffers are incomplete.  Call this after the stream has been synchronised: it reads the flag
+ * (a blocking 4-byte copy), clears it, and returns BCAST_ERR_TIMEOUT if it was set, else BCAST_OK.
+ * The other executors have no waits and never set it.
  */
 int bcast_exec_status(const bcast_plan_t *plan);
 

@@ -405,7 +405,7 @@ int launch_walk(const bcast_plan_t &p, const bcast_device_state &ds, void *const
 int launch_walk_bulk(const bcast_plan_t &p, const bcast_device_state &ds, void *const *rank_bufs, cudaStream_t st,
                      unsigned long long *trace)
 {
-    WalkDev w = walk_dev(p, ds, false, ds.d_reg_slices, ds.n_reg, trace);
+    WalkDev w = walk_dev(p, ds, env_int("BCAST_BULK_PLAN_ORDER", 0) != 0, ds.d_reg_slices, ds.n_reg, trace);
     BulkDev b{ds.d_bulk_slices, ds.n_bulk, ds.bulk_spin_limit, ds.d_status};
     return launch_with_ptrs(bulk_kernel(p.P, trace != nullptr), dim3(ds.bulk_grid), dim3(kBulkThreads),
                             (size_t)kBulkWorkers * kBulkSeg, st, rank_bufs, p.P, trace != nullptr, {&w, &b});

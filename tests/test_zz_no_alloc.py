@@ -80,3 +80,48 @@ def test_static_refuses_plans_beyond_its_capacity():
     torch.cuda.synchronize()
     assert not dev.any()                                  # nothing was launched
     assert "scratch" in B.bcast_strerror(B.BCAST_ERR_CAPACITY)
+
+
+def test_static_allocates_no_device_memory():
+    # the property the entry point exists for: on a plan that bcast_exec never saw (so no cached
+    # device tables can stand in), the driver's count of free device memory must not move
+    wl = W.Workload("static_noalloc", 24, 3, 3 * W.MiB + 7, 43)
+    msg = W.message_bytes(wl.seed, wl.nbytes)
+    bufs = RankBuffers(wl.P, wl.root, wl.nbytes, msg)
+    st = torch.cuda.current_stream()
+    warm = B.bcast_plan(wl.P, wl.root, wl.nbytes, B.BCAST_NATIVE)       # module and kernel loading happen here
+    B.bcast_exec_static(bufs.pointers(), warm, st)
+    torch.cuda.synchronize()
+    bufs.reset()
+    fresh = B.bcast_plan(wl.P, wl.root, wl.nbytes, B.BCAST_TUNED)
+    torch.cuda.synchronize()
+    free_before = torch.cuda.mem_get_info()[0]
+    B.bcast_exec_static(bufs.pointers(), fresh, st)
+    B.bcast_exec_static(bufs.pointers(), fresh, st)
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free_before
+    B.bcast_exec_status(fresh)                                         # no device state was created for this plan
+    assert bufs.all_equal_message() and bufs.guards_intact()
+
+
+def test_static_refuses_a_capturing_stream():
+    # its copy into the shared array must not be recorded into a graph: the call says so instead
+    wl = W.Workload("static_capture", 8, 0, 65536, 44)
+    bufs = RankBuffers(wl.P, wl.root, wl.nbytes, W.message_bytes(wl.seed, wl.nbytes))
+    plan = B.bcast_plan(wl.P, wl.root, wl.nbytes, B.BCAST_TUNED)
+    B.bcast_exec_static(bufs.pointers(), plan, torch.cuda.current_stream())   # first call on the device: outside capture
+    torch.cuda.synchronize()
+    bufs.reset()
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    code = None
+    with torch.cuda.graph(graph, stream=side):
+        try:
+            B.bcast_exec_static(bufs.pointers(), plan, side)
+        except B.BcastError as e:
+            code = e.code
+    assert code == B.BCAST_ERR_INVAL
+    torch.cuda.synchronize()
+    B.bcast_exec_static(bufs.pointers(), plan, torch.cuda.current_stream())   # still usable afterwards
+    torch.cuda.synchronize()
+    assert bufs.all_equal_message() and bufs.guards_intact()
