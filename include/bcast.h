@@ -311,6 +311,80 @@ int bcast_exec_traced(void *const *rank_bufs, const bcast_plan_t *plan, void *cu
                       uint64_t *device_msg_bytes);
 
 /*
+ * ---- The ranks of a plan spread over several GPUs of one NVLink/NVSwitch domain ----------------
+ * (Section V measures the broadcast where ring neighbours sit on different nodes; here the P ranks
+ * are dealt to G GPUs and a message whose source and destination are on different GPUs crosses
+ * NVLink.)  Every rank's buffer lives in the memory of the GPU that owns the rank.  A message is
+ * performed by the GPU that owns its destination rank: its kernel loads from the source rank's
+ * buffer -- local memory or a peer's, by ordinary peer loads, never a multicast load -- and stores
+ * into its own memory.  The work is cut into phases: a hop (message restricted to one chunk) whose
+ * source copy was written by another GPU runs one phase after the hop that wrote it; hops inside one
+ * GPU keep the order of the one-GPU walk.  Phase k+1 of every GPU is ordered after phase k of all
+ * GPUs, by CUDA events between streams (bcast_shard_exec, one process drives all GPUs) or by whatever
+ * barrier the caller has between processes (bcast_shard_exec_phase, one process per GPU).  No kernel
+ * ever waits for another kernel.
+ */
+typedef struct bcast_shard bcast_shard_t; /* opaque; created and freed by the library */
+
+/*
+ * bcast_shard_create -- partition a plan over num_gpus GPUs.  Host only; needs no GPU.
+ *   plan      must outlive the partition
+ *   num_gpus  1..P
+ *   rank_gpu  HOST array [P]: the GPU (0..num_gpus-1) that owns each absolute rank, or NULL for
+ *             contiguous groups (rank r on GPU floor(r * num_gpus / P))
+ * Errors: BCAST_ERR_INVAL, BCAST_ERR_NOMEM.
+ */
+int bcast_shard_create(const bcast_plan_t *plan, int num_gpus, const int32_t *rank_gpu, bcast_shard_t **out);
+/* Release a partition and its device tables.  NULL is ignored. */
+void bcast_shard_free(bcast_shard_t *shard);
+
+/* Read-only views; HOST pointers owned by the partition. */
+int32_t bcast_shard_num_gpus(const bcast_shard_t *shard);
+int32_t bcast_shard_num_phases(const bcast_shard_t *shard);          /* 0 for a plan that moves nothing */
+const int32_t *bcast_shard_rank_gpu(const bcast_shard_t *shard);     /* [P]                                */
+const int32_t *bcast_shard_msg_gpu(const bcast_shard_t *shard);      /* [num_xfers]: GPU that performs it  */
+/* [num_xfers]: the phase of a message's hops; last = 0 gives the earliest, last != 0 the latest (they
+   differ only for a message whose chunks reached its source in different phases); -1 for a message
+   that moves nothing */
+const int32_t *bcast_shard_msg_phase(const bcast_shard_t *shard, int last);
+/* Bytes (sum of len) and number of the messages whose source and destination ranks are on different
+   GPUs: what crosses NVLink.  The tuned ring saves here exactly what it saves in total. */
+uint64_t bcast_shard_crossing_bytes(const bcast_shard_t *shard);
+int64_t bcast_shard_crossing_msgs(const bcast_shard_t *shard);
+/* The messages (indices into bcast_plan_xfers) that GPU `gpu` performs in phase `phase` on the bytes
+   of relative chunk `chunk`, in execution order; two-call protocol like bcast_plan_walk_order. */
+int64_t bcast_shard_hops(const bcast_shard_t *shard, int phase, int gpu, int chunk, int64_t *out, int64_t cap);
+
+/*
+ * bcast_shard_exec -- perform the whole plan from one process that drives all GPUs.
+ *   rank_bufs     HOST array of P DEVICE pointers; rank r's buffer must be memory of device
+ *                 gpu_device[rank_gpu[r]] (peer access between those devices enabled by the caller
+ *                 where they differ); alignment and disjointness as for bcast_exec
+ *   gpu_device    HOST array [num_gpus]: CUDA device ordinal of every GPU of the partition (they may
+ *                 repeat: several, or all, "GPUs" of the partition on one device); fixed by the first call
+ *   cuda_streams  HOST array [num_gpus] of cudaStream_t, stream g on device gpu_device[g]; streams of
+ *                 GPUs mapped to one device may be the same stream or different ones.  The message
+ *                 must be in rank_bufs[root] before the work enqueued here starts on the root's GPU
+ *                 (enqueue its copy on that GPU's stream, or synchronise first).
+ *   device_msg_bytes  NULL, or counters as for bcast_exec_traced, reachable from every device used
+ * Asynchronous: when all the streams have been synchronised, every rank buffer holds the message.
+ * The first call builds device tables (cudaMalloc) on every device.  Errors: as bcast_exec.
+ */
+int bcast_shard_exec(bcast_shard_t *shard, void *const *rank_bufs, const int *gpu_device, void *const *cuda_streams,
+                     uint64_t *device_msg_bytes);
+
+/*
+ * bcast_shard_exec_phase -- enqueue only GPU `gpu`'s kernel of phase `phase`, on the current device
+ * and the given stream: the building block for one process per GPU.  The caller runs the phases in
+ * ascending order and makes sure that phase k of every GPU has completed before any GPU starts phase
+ * k+1 (stream synchronisation plus a barrier between the processes); rank_bufs holds, for ranks owned
+ * by other GPUs, pointers through which this device can read their buffers (peer or IPC mappings).
+ * A (phase, gpu) pair without work enqueues nothing.  Errors: as bcast_exec.
+ */
+int bcast_shard_exec_phase(bcast_shard_t *shard, void *const *rank_bufs, int phase, int gpu, void *cuda_stream,
+                           uint64_t *device_msg_bytes);
+
+/*
  * bcast_exec_status -- did a kernel of this plan give up on a bounded wait?
  * The bulk-copy kernel (BCAST_EXEC_WALK_BULK) polls an mbarrier for the arrival of every load; the
  * number of polls is limited, so that a copy that never completes ends the kernel instead of

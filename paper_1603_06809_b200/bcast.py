@@ -39,6 +39,9 @@ SYMBOLS = (
     "bcast_plan_xfers", "bcast_plan_step_begin", "bcast_plan_bytes_sent", "bcast_plan_bytes_recv",
     "bcast_plan_msgs_sent", "bcast_plan_msgs_recv", "bcast_plan_total_bytes", "bcast_plan_walk_order",
     "bcast_plan_walk_pairing", "bcast_plan_walk_slices", "bcast_exec_traced", "bcast_exec",
+    "bcast_shard_create", "bcast_shard_free", "bcast_shard_num_gpus", "bcast_shard_num_phases", "bcast_shard_rank_gpu",
+    "bcast_shard_msg_gpu", "bcast_shard_msg_phase", "bcast_shard_crossing_bytes", "bcast_shard_crossing_msgs",
+    "bcast_shard_hops", "bcast_shard_exec", "bcast_shard_exec_phase",
     "bcast_exec_mode", "bcast_exec_host", "bcast_exec_static", "bcast_exec_status", "bcast_exec_num_launches", "bcast_strerror",
     "bcast_last_cuda_error",
 )
@@ -60,6 +63,14 @@ _sig = {
     "bcast_plan_walk_slices": (_i64, [_vp, _i, ctypes.POINTER(ctypes.c_int64), _i64]),
     "bcast_exec_traced": (_i, [_vpp, _vp, _vp, _i, _vp]),
     "bcast_exec": (_i, [_vpp, _vp, _vp]),
+    "bcast_shard_create": (_i, [_vp, _i, ctypes.POINTER(ctypes.c_int32), _vpp]),
+    "bcast_shard_free": (None, [_vp]),
+    "bcast_shard_num_gpus": (_i32, [_vp]), "bcast_shard_num_phases": (_i32, [_vp]),
+    "bcast_shard_rank_gpu": (_vp, [_vp]), "bcast_shard_msg_gpu": (_vp, [_vp]), "bcast_shard_msg_phase": (_vp, [_vp, _i]),
+    "bcast_shard_crossing_bytes": (_u64, [_vp]), "bcast_shard_crossing_msgs": (_i64, [_vp]),
+    "bcast_shard_hops": (_i64, [_vp, _i, _i, _i, ctypes.POINTER(ctypes.c_int64), _i64]),
+    "bcast_shard_exec": (_i, [_vp, _vpp, ctypes.POINTER(ctypes.c_int), _vpp, _vp]),
+    "bcast_shard_exec_phase": (_i, [_vp, _vpp, _i, _i, _vp, _vp]),
     "bcast_exec_mode": (_i, [_vpp, _vp, _vp, _i]),
     "bcast_exec_host": (_i, [_vpp, _vp, _vp, _i, _vp, _vpp]),
     "bcast_exec_static": (_i, [_vpp, _vp, _vp]),
@@ -292,3 +303,98 @@ def bcast_strerror(code: int) -> str:
 
 def bcast_last_cuda_error() -> int:
     return _lib.bcast_last_cuda_error()
+
+
+# ---- the ranks of a plan spread over several GPUs
+class Shard:
+    """Owner of a ``bcast_shard_t*``; keeps its plan alive."""
+
+    def __init__(self, handle: int, plan: Plan):
+        self._h = ctypes.c_void_p(handle)
+        self.plan = plan
+
+    @property
+    def handle(self) -> ctypes.c_void_p:
+        if not self._h:
+            raise ValueError("partition already freed")
+        return self._h
+
+    def free(self) -> None:
+        if self._h:
+            _lib.bcast_shard_free(self._h)
+            self._h = ctypes.c_void_p(None)
+
+    def __del__(self):
+        try:
+            self.free()
+        except Exception:
+            pass
+
+
+def bcast_shard_create(plan: Plan, num_gpus: int, rank_gpu=None) -> Shard:
+    arr = None
+    if rank_gpu is not None:
+        if len(rank_gpu) != bcast_plan_num_ranks(plan):
+            raise BcastError(BCAST_ERR_INVAL, "bcast_shard_create (len(rank_gpu) != P)")
+        arr = (ctypes.c_int32 * len(rank_gpu))(*[int(g) for g in rank_gpu])
+    out = ctypes.c_void_p(None)
+    _check(_lib.bcast_shard_create(plan.handle, num_gpus, arr, ctypes.byref(out)), "bcast_shard_create")
+    return Shard(out.value, plan)
+
+
+def bcast_shard_free(shard: Shard) -> None:
+    shard.free()
+
+
+def bcast_shard_num_gpus(shard: Shard) -> int: return _lib.bcast_shard_num_gpus(shard.handle)
+def bcast_shard_num_phases(shard: Shard) -> int: return _lib.bcast_shard_num_phases(shard.handle)
+def bcast_shard_crossing_bytes(shard: Shard) -> int: return _lib.bcast_shard_crossing_bytes(shard.handle)
+def bcast_shard_crossing_msgs(shard: Shard) -> int: return _lib.bcast_shard_crossing_msgs(shard.handle)
+
+
+def bcast_shard_rank_gpu(shard: Shard) -> np.ndarray:
+    return _view(_lib.bcast_shard_rank_gpu(shard.handle), bcast_plan_num_ranks(shard.plan), np.int32)
+
+
+def bcast_shard_msg_gpu(shard: Shard) -> np.ndarray:
+    return _view(_lib.bcast_shard_msg_gpu(shard.handle), bcast_plan_num_xfers(shard.plan), np.int32)
+
+
+def bcast_shard_msg_phase(shard: Shard, last: bool = False) -> np.ndarray:
+    return _view(_lib.bcast_shard_msg_phase(shard.handle, int(last)), bcast_plan_num_xfers(shard.plan), np.int32)
+
+
+def bcast_shard_hops(shard: Shard, phase: int, gpu: int, chunk: int) -> np.ndarray:
+    n = _lib.bcast_shard_hops(shard.handle, phase, gpu, chunk, None, 0)
+    if n < 0:
+        raise BcastError(int(n), "bcast_shard_hops")
+    out = np.zeros(int(n), dtype=np.int64)
+    if n:
+        got = _lib.bcast_shard_hops(shard.handle, phase, gpu, chunk, out.ctypes.data_as(ctypes.POINTER(ctypes.c_int64)), int(n))
+        assert got == n
+    return out
+
+
+def _counter_ptr(device_msg_bytes) -> ctypes.c_void_p:
+    if device_msg_bytes is None:
+        return ctypes.c_void_p(None)
+    return ctypes.c_void_p(device_msg_bytes.data_ptr() if hasattr(device_msg_bytes, "data_ptr") else int(device_msg_bytes))
+
+
+def bcast_shard_exec(shard: Shard, rank_bufs, gpu_device, streams, device_msg_bytes=None) -> None:
+    """``gpu_device``: CUDA device ordinal per GPU of the partition; ``streams``: one stream per GPU
+    (torch streams or raw handles)."""
+    G = bcast_shard_num_gpus(shard)
+    if len(rank_bufs) != bcast_plan_num_ranks(shard.plan) or len(gpu_device) != G or len(streams) != G:
+        raise BcastError(BCAST_ERR_INVAL, "bcast_shard_exec (array lengths)")
+    devs = (ctypes.c_int * G)(*[int(d) for d in gpu_device])
+    sts = (ctypes.c_void_p * G)(*[_stream_ptr(s).value for s in streams])
+    _check(_lib.bcast_shard_exec(shard.handle, _ptr_array(rank_bufs, "rank_bufs"), devs, sts, _counter_ptr(device_msg_bytes)),
+           "bcast_shard_exec")
+
+
+def bcast_shard_exec_phase(shard: Shard, rank_bufs, phase: int, gpu: int, stream=None, device_msg_bytes=None) -> None:
+    if len(rank_bufs) != bcast_plan_num_ranks(shard.plan):
+        raise BcastError(BCAST_ERR_INVAL, "bcast_shard_exec_phase (len(rank_bufs) != P)")
+    _check(_lib.bcast_shard_exec_phase(shard.handle, _ptr_array(rank_bufs, "rank_bufs"), phase, gpu, _stream_ptr(stream),
+                                       _counter_ptr(device_msg_bytes)), "bcast_shard_exec_phase")

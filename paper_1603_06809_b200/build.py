@@ -12,8 +12,8 @@ import sys
 PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 REPO_DIR = os.path.dirname(PKG_DIR)
 LIB_PATH = os.path.join(PKG_DIR, "libbcast_b200.so")
-SOURCES = [os.path.join(PKG_DIR, "csrc", f) for f in ("plan.cpp", "walk_tables.cpp", "exec.cu")]
-HEADERS = [os.path.join(REPO_DIR, "include", "bcast.h")] + [os.path.join(PKG_DIR, "csrc", f) for f in ("plan_internal.h", "walk_tables.h", "kernels.cuh")]
+SOURCES = [os.path.join(PKG_DIR, "csrc", f) for f in ("plan.cpp", "walk_tables.cpp", "shard.cpp", "exec.cu")]
+HEADERS = [os.path.join(REPO_DIR, "include", "bcast.h")] + [os.path.join(PKG_DIR, "csrc", f) for f in ("plan_internal.h", "walk_tables.h", "exec_internal.h", "kernels.cuh")]
 
 NVCC_FLAGS = [
     "-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",

@@ -10,6 +10,7 @@
 #include <new>
 #include <vector>
 
+#include "exec_internal.h"
 #include "kernels.cuh"
 #include "plan_internal.h"
 #include "walk_tables.h"
@@ -213,7 +214,7 @@ struct WalkShape {
     int u = 1, grid = 1;
 };
 
-int choose_walk_shape(const bcast_plan_t &p, int sm_count, WalkShape *shape)
+int choose_shape(bool few_hops, const std::function<long long(int)> &slices_for, int P, int sm_count, WalkShape *shape)
 {
     const int forced_u = env_int("BCAST_WALK_WORDS", 0);
     const int forced_bps = env_int("BCAST_WALK_BLOCKS_PER_SM", 0);
@@ -221,19 +222,19 @@ int choose_walk_shape(const bcast_plan_t &p, int sm_count, WalkShape *shape)
     int rc, resident = 1, u = 0, bps = 0;
     if (u_ok || forced_bps > 0) {
         u = u_ok ? forced_u : kMaxWords;
-        if ((rc = walk_blocks_per_sm(u, p.P, &resident))) return rc;
+        if ((rc = walk_blocks_per_sm(u, P, &resident))) return rc;
         bps = forced_bps > 0 ? std::min(forced_bps, resident) : resident;
-    } else if (p.P <= 4) {
-        u = p.P <= 3 ? 4 : 2;
-        if ((rc = walk_blocks_per_sm(u, p.P, &resident))) return rc;
+    } else if (few_hops) {
+        u = P <= 3 ? 4 : 2;
+        if ((rc = walk_blocks_per_sm(u, P, &resident))) return rc;
         bps = resident;
-    } else if (count_slices(p, 512ull * kMaxWords, true) * 5 > (long long)sm_count * kWarpsPerBlock * 7) {   // > 1.4 rounds
+    } else if (slices_for(kMaxWords) * 5 > (long long)sm_count * kWarpsPerBlock * 7) {   // > 1.4 rounds
         u = kMaxWords;
         bps = 1;
     } else {
         for (int cand = 1; cand <= kMaxWords; cand++) {
-            if ((rc = walk_blocks_per_sm(cand, p.P, &resident))) return rc;
-            const long long slices = count_slices(p, 512ull * cand, true);
+            if ((rc = walk_blocks_per_sm(cand, P, &resident))) return rc;
+            const long long slices = slices_for(cand);
             if (slices <= (long long)sm_count * resident * kWarpsPerBlock) {
                 u = cand;
                 bps = (int)std::max<long long>(1, (slices + (long long)sm_count * kWarpsPerBlock - 1) /
@@ -243,17 +244,24 @@ int choose_walk_shape(const bcast_plan_t &p, int sm_count, WalkShape *shape)
         }
         if (!u) { u = kMaxWords; bps = 1; }
     }
-    const long long slices = std::max<long long>(1, count_slices(p, 512ull * u, true));
+    const long long slices = std::max<long long>(1, slices_for(u));
     shape->u = u;
     shape->grid = (int)std::min<long long>(slices, (long long)sm_count * std::max(1, bps));
     return BCAST_OK;
 }
 
+int choose_walk_shape(const bcast_plan_t &p, int sm_count, WalkShape *shape)
+{
+    return choose_shape(p.P <= 4, [&](int u) { return count_slices(p, 512ull * u, true, nullptr); }, p.P, sm_count, shape);
+}
+
 // Hop lists and dual lists, then the slices of the register walk for the chosen shape.
 int build_walk_tables(const bcast_plan_t &p, bcast_device_state &ds)
 {
+    HopLists lists;
+    whole_plan_hops(p, lists);
     WalkTables t;
-    make_walk_tables(p, t);
+    make_walk_tables(p, lists, t);
     int rc;
     if ((rc = upload(&ds.d_hops, t.hops))) return rc;
     if ((rc = upload(&ds.d_hops_plan, t.hops_plan))) return rc;
@@ -269,7 +277,7 @@ int build_walk_tables(const bcast_plan_t &p, bcast_device_state &ds)
     ds.walk_u = shape.u;
     ds.walk_grid = shape.grid;
     std::vector<WalkSlice> slices;
-    make_slices(p, 512ull * ds.walk_u, env_int("BCAST_WALK_DUAL", 1) != 0, slices);
+    make_slices(p, 512ull * ds.walk_u, env_int("BCAST_WALK_DUAL", 1) != 0, nullptr, slices);
     ds.n_slices = (long long)slices.size();
     return upload(&ds.d_slices, slices);
 }
@@ -498,6 +506,33 @@ int exec_checked(void *const *rank_bufs, const bcast_plan_t *plan, void *cuda_st
 
 }  // namespace
 
+// ======================================================================================= for shard.cpp
+int bcast_internal_walk_shape(bool few_hops, const std::function<long long(int)> &slices_for, int P, int sm_count, int *u,
+                              int *grid)
+{
+    WalkShape shape;
+    const int rc = choose_shape(few_hops, slices_for, P, sm_count, &shape);
+    *u = shape.u;
+    *grid = shape.grid;
+    return rc;
+}
+
+int bcast_internal_launch_walk(const WalkDev &w, int u, int grid, void *const *rank_bufs, int P, void *cuda_stream)
+{
+    WalkDev copy = w;
+    const bool trace = w.trace != nullptr;
+    return launch_with_ptrs(walk_kernel(u, P, trace), dim3(grid), dim3(kThreads), 0, (cudaStream_t)cuda_stream, rank_bufs, P,
+                            trace, {&copy});
+}
+
+int bcast_internal_validate_bufs(void *const *rank_bufs, size_t P, uint64_t nbytes) { return validate_bufs(rank_bufs, P, nbytes); }
+
+int bcast_internal_cuda_failed(int cuda_error)
+{
+    t_last_cuda_error = cuda_error;
+    return cuda_error == (int)cudaErrorMemoryAllocation ? BCAST_ERR_NOMEM : BCAST_ERR_CUDA;
+}
+
 // ======================================================================================= C ABI
 extern "C" {
 
@@ -588,8 +623,8 @@ int64_t bcast_plan_walk_slices(const bcast_plan_t *plan, int words, int64_t *out
     if (!plan || words < 1 || words > kMaxWords || cap < 0 || (cap > 0 && !out)) return BCAST_ERR_INVAL;
     try {
         std::vector<WalkSlice> slices;
-        if (plan->total_bytes) make_slices(*plan, 512ull * words, true, slices);
-        if ((long long)slices.size() != (plan->total_bytes ? count_slices(*plan, 512ull * words, true) : 0))
+        if (plan->total_bytes) make_slices(*plan, 512ull * words, true, nullptr, slices);
+        if ((long long)slices.size() != (plan->total_bytes ? count_slices(*plan, 512ull * words, true, nullptr) : 0))
             return BCAST_ERR_INVAL;                       // the two must agree: the launch shape relies on it
         for (int64_t i = 0; i < (int64_t)slices.size() && i < cap; i++) {
             out[3 * i] = slices[i].seg;
@@ -685,14 +720,16 @@ int make_static_image(const bcast_plan_t &p, int sm_count, bcast_static_image &i
     WalkShape shape;
     int rc = choose_walk_shape(p, sm_count, &shape);
     if (rc) return rc;
+    HopLists lists;
+    whole_plan_hops(p, lists);
     WalkTables t;
-    make_walk_tables(p, t);
+    make_walk_tables(p, lists, t);
     std::vector<WalkSlice> slices;
     for (int attempt = 0; attempt < 4; attempt++) {
         const bool use_dual = (attempt & 1) == 0;
         const int u = attempt < 2 ? shape.u : kMaxWords;
         if (attempt >= 2 && shape.u == kMaxWords) break;
-        make_slices(p, 512ull * u, use_dual, slices);
+        make_slices(p, 512ull * u, use_dual, nullptr, slices);
         const size_t dual_bytes = use_dual ? t.dual.size() * sizeof(DualSlot) : 0;
         img.off_dual_begin = round256(t.hop_begin.size() * sizeof(int));
         img.off_slices = img.off_dual_begin + round256(t.dual_begin.size() * sizeof(int));

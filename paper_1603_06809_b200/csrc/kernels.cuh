@@ -50,19 +50,6 @@ struct DevXfer {      // one message, device copy (STEPS executor)
     uint32_t pad;
 };
 
-struct WalkDev {      // device tables of one WALK launch
-    const WalkSlice *slices;
-    long long n_slices;
-    const uint32_t *hops;        // per chunk, the order in use
-    const int *hop_begin;
-    const DualSlot *dual;        // per chunk boundary
-    const int *dual_begin;
-    const int32_t *hop_msg;      // TRACE: plan message of every hop / slot
-    const DualMsg *dual_msg;
-    unsigned long long *trace;   // TRACE: bytes stored per plan message
-    uint64_t scatter_size, nbytes;
-};
-
 // ---- memory operations.  volatile + "memory": the compiler must keep loads and stores of
 // successive hops in program order, because a hop may read what the previous hop wrote.
 __device__ __forceinline__ uint4 ld16(const uint8_t *p)

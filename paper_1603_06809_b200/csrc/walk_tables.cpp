@@ -12,21 +12,24 @@ inline uint32_t encode_hop(const bcast_plan_t &p, int64_t i)
     return (uint32_t)p.xfers[i].src_rank | ((uint32_t)p.xfers[i].dst_rank << 16);
 }
 
+inline bool is_active(const std::vector<char> *active, uint64_t c) { return !active || (*active)[(size_t)c] != 0; }
+
 // Classify segment g of the `seg`-byte grid and append its slice(s).
-void classify_segment(const bcast_plan_t &p, uint64_t seg, uint64_t g, bool use_dual, std::vector<WalkSlice> &ragged,
-                      std::vector<WalkSlice> &dual, std::vector<WalkSlice> &full)
+void classify_segment(const bcast_plan_t &p, uint64_t seg, uint64_t g, bool use_dual, const std::vector<char> *active,
+                      std::vector<WalkSlice> &ragged, std::vector<WalkSlice> &dual, std::vector<WalkSlice> &full)
 {
     const uint64_t lo = g * seg, hi = std::min(lo + seg, p.nbytes);
     if (lo >= hi || p.S == 0) return;
     const uint64_t c0 = lo / p.S, c1 = (hi - 1) / p.S;      // chunks that overlap the segment: all non-empty
     const bool whole = hi == lo + seg;
     if (c0 == c1) {
-        (whole ? full : ragged).push_back(WalkSlice{(uint32_t)g, (uint32_t)c0 | ((whole ? kSliceFull : kSliceRagged) << kSliceKindShift)});
-    } else if (c1 == c0 + 1 && whole && use_dual) {
+        if (is_active(active, c0))
+            (whole ? full : ragged).push_back(WalkSlice{(uint32_t)g, (uint32_t)c0 | ((whole ? kSliceFull : kSliceRagged) << kSliceKindShift)});
+    } else if (c1 == c0 + 1 && whole && use_dual && is_active(active, c0) && is_active(active, c1)) {
         dual.push_back(WalkSlice{(uint32_t)g, (uint32_t)c0 | (kSliceDual << kSliceKindShift)});
     } else {
         for (uint64_t c = c0; c <= c1; c++)
-            ragged.push_back(WalkSlice{(uint32_t)g, (uint32_t)c | (kSliceRagged << kSliceKindShift)});
+            if (is_active(active, c)) ragged.push_back(WalkSlice{(uint32_t)g, (uint32_t)c | (kSliceRagged << kSliceKindShift)});
     }
 }
 
@@ -111,19 +114,22 @@ void pair_hops(const bcast_plan_t &p, const std::vector<int64_t> &lower, const s
     }
 }
 
-void make_walk_tables(const bcast_plan_t &p, WalkTables &t)
+void whole_plan_hops(const bcast_plan_t &p, HopLists &lists)
+{
+    messages_by_chunk(p, lists.plan_order);
+    lists.walk_order.assign(p.P, {});
+    for (int c = 0; c < p.P; c++) order_by_dependency(p, lists.plan_order[c], lists.walk_order[c]);
+}
+
+void make_walk_tables(const bcast_plan_t &p, const HopLists &lists, WalkTables &t)
 {
     const int P = p.P;
-    std::vector<std::vector<int64_t>> per_chunk;
-    messages_by_chunk(p, per_chunk);
     t.hop_begin.assign(P + 1, 0);
     t.hops.clear(); t.hops_plan.clear(); t.hop_msg.clear(); t.hop_msg_plan.clear();
-    std::vector<int64_t> reordered;
     for (int c = 0; c < P; c++) {
         t.hop_begin[c] = (int)t.hops.size();
-        order_by_dependency(p, per_chunk[c], reordered);
-        for (int64_t i : reordered) { t.hops.push_back(encode_hop(p, i)); t.hop_msg.push_back((int32_t)i); }
-        for (int64_t i : per_chunk[c]) { t.hops_plan.push_back(encode_hop(p, i)); t.hop_msg_plan.push_back((int32_t)i); }
+        for (int64_t i : lists.walk_order[c]) { t.hops.push_back(encode_hop(p, i)); t.hop_msg.push_back((int32_t)i); }
+        for (int64_t i : lists.plan_order[c]) { t.hops_plan.push_back(encode_hop(p, i)); t.hop_msg_plan.push_back((int32_t)i); }
     }
     t.hop_begin[P] = (int)t.hops.size();
 
@@ -132,8 +138,8 @@ void make_walk_tables(const bcast_plan_t &p, WalkTables &t)
     std::vector<DualMsg> slots;
     for (int c = 0; c < P; c++) {
         t.dual_begin[c] = (int)t.dual.size();
-        if (c + 1 >= P || per_chunk[c].empty() || per_chunk[c + 1].empty()) continue;
-        pair_hops(p, per_chunk[c], per_chunk[c + 1], slots);
+        if (c + 1 >= P || lists.plan_order[c].empty() || lists.plan_order[c + 1].empty()) continue;
+        pair_hops(p, lists.plan_order[c], lists.plan_order[c + 1], slots);
         const size_t first = t.dual.size();
         for (const DualMsg &s : slots) {
             t.dual.push_back(DualSlot{s.a < 0 ? kNoHop : encode_hop(p, s.a), s.b < 0 ? kNoHop : encode_hop(p, s.b)});
@@ -151,12 +157,12 @@ void make_walk_tables(const bcast_plan_t &p, WalkTables &t)
     t.dual_begin[P] = (int)t.dual.size();
 }
 
-void make_slices(const bcast_plan_t &p, uint64_t seg_bytes, bool use_dual, std::vector<WalkSlice> &slices)
+void make_slices(const bcast_plan_t &p, uint64_t seg_bytes, bool use_dual, const std::vector<char> *active,
+                 std::vector<WalkSlice> &slices)
 {
     std::vector<WalkSlice> ragged, dual, full;
     const uint64_t nseg = (p.nbytes + seg_bytes - 1) / seg_bytes;
-    full.reserve((size_t)nseg);
-    for (uint64_t g = 0; g < nseg; g++) classify_segment(p, seg_bytes, g, use_dual, ragged, dual, full);
+    for (uint64_t g = 0; g < nseg; g++) classify_segment(p, seg_bytes, g, use_dual, active, ragged, dual, full);
     slices.clear();
     slices.reserve(ragged.size() + dual.size() + full.size());
     slices.insert(slices.end(), ragged.begin(), ragged.end());
@@ -164,10 +170,16 @@ void make_slices(const bcast_plan_t &p, uint64_t seg_bytes, bool use_dual, std::
     slices.insert(slices.end(), full.begin(), full.end());
 }
 
-long long count_slices(const bcast_plan_t &p, uint64_t seg_bytes, bool use_dual)
+long long count_slices(const bcast_plan_t &p, uint64_t seg_bytes, bool use_dual, const std::vector<char> *active)
 {
-    // every segment is one slice, except those that are cut into ragged slices per chunk
     if (p.nbytes == 0 || p.S == 0) return 0;
+    if (active) {                                   // a partial walk: count what make_slices would make
+        std::vector<WalkSlice> ragged, dual, full;
+        const uint64_t nseg = (p.nbytes + seg_bytes - 1) / seg_bytes;
+        for (uint64_t g = 0; g < nseg; g++) classify_segment(p, seg_bytes, g, use_dual, active, ragged, dual, full);
+        return (long long)(ragged.size() + dual.size() + full.size());
+    }
+    // every segment is one slice, except those that are cut into ragged slices per chunk
     const uint64_t nseg = (p.nbytes + seg_bytes - 1) / seg_bytes;
     long long n = (long long)nseg;
     for (int c = 1; c < p.P; c++) {
@@ -200,7 +212,7 @@ void make_bulk_slices(const bcast_plan_t &p, uint64_t bulk_seg, uint64_t reg_seg
             continue;
         }
         for (uint64_t q = g * per; q < (g + 1) * per && q * reg_seg < p.nbytes; q++)
-            classify_segment(p, reg_seg, q, true, ragged, dual, full);
+            classify_segment(p, reg_seg, q, true, nullptr, ragged, dual, full);
     }
     reg.insert(reg.end(), ragged.begin(), ragged.end());
     reg.insert(reg.end(), dual.begin(), dual.end());

@@ -36,6 +36,27 @@ struct DualMsg {       // indices into the plan's message array, -1 where the sl
     int32_t a, b;
 };
 
+// Device pointers of the tables one WALK launch reads (filled by the host, passed by value).
+struct WalkDev {
+    const WalkSlice *slices;
+    long long n_slices;
+    const uint32_t *hops;        // per chunk, the order in use
+    const int *hop_begin;
+    const DualSlot *dual;        // per chunk boundary
+    const int *dual_begin;
+    const int32_t *hop_msg;      // traced launches only: plan message of every hop / slot
+    const DualMsg *dual_msg;
+    unsigned long long *trace;   // traced launches only: bytes stored per plan message
+    uint64_t scatter_size, nbytes;
+};
+
+// Per relative chunk, the plan messages ("hops") a walk performs on the bytes of that chunk: in
+// the order the full and ragged slices take them, and in plan order (what the dual lists are
+// merged from).  A walk over a part of the plan (one GPU's share of one phase) has shorter lists.
+struct HopLists {
+    std::vector<std::vector<int64_t>> walk_order, plan_order;
+};
+
 struct WalkTables {
     // per relative chunk c: hops [hop_begin[c], hop_begin[c+1]) in dependency order / plan order,
     // and beside every hop the index of the plan message it performs
@@ -61,17 +82,23 @@ void order_by_dependency(const bcast_plan_t &p, const std::vector<int64_t> &plan
 void pair_hops(const bcast_plan_t &p, const std::vector<int64_t> &lower, const std::vector<int64_t> &upper,
                std::vector<DualMsg> &slots);
 
-// Hop lists and dual lists of a plan (independent of the segment size).
-void make_walk_tables(const bcast_plan_t &p, WalkTables &t);
+// The hop lists of the whole plan: plan order, and level order of the dependency tree where legal.
+void whole_plan_hops(const bcast_plan_t &p, HopLists &lists);
+
+// Device-table images (hop lists and dual lists) from hop lists; independent of the segment size.
+void make_walk_tables(const bcast_plan_t &p, const HopLists &lists, WalkTables &t);
 
 // The slices of the message for segments of `seg_bytes` bytes, restricted to segments
 // [seg_first, seg_last) (pass 0, UINT64_MAX for all).  Order: ragged slices first, then dual
 // slices, then full slices, each group in message order (the slow kinds start first).
 // `use_dual` = false cuts every segment that holds a boundary into ragged slices instead.
-void make_slices(const bcast_plan_t &p, uint64_t seg_bytes, bool use_dual, std::vector<WalkSlice> &slices);
+// `active` (NULL: all): per relative chunk, whether the walk has any hop for it; bytes of inactive
+// chunks get no slice, and a boundary segment is a dual slice only if both its chunks are active.
+void make_slices(const bcast_plan_t &p, uint64_t seg_bytes, bool use_dual, const std::vector<char> *active,
+                 std::vector<WalkSlice> &slices);
 
 // Number of slices make_slices() would produce.
-long long count_slices(const bcast_plan_t &p, uint64_t seg_bytes, bool use_dual);
+long long count_slices(const bcast_plan_t &p, uint64_t seg_bytes, bool use_dual, const std::vector<char> *active);
 
 // Slices of the bulk-copy walk: every whole 16 KiB segment inside one chunk is a bulk slice (kind
 // kSliceFull on the 16 KiB grid); the other 16 KiB segments are cut on the 4 KiB grid into
