@@ -48,6 +48,11 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg4", help="cfg1..cfg4, or P<ranks>x<bytes>[r<root>] (root defaults to P-1)")
     ap.add_argument("--cold", action="store_true", help="flush L2 between the timed broadcasts")
+    ap.add_argument("--sharded", action="store_true",
+                    help="with --gpus N under torchrun: ONE broadcast whose P ranks are spread over the N GPUs "
+                         "(each process owns its GPU's rank buffers; phases separated by barriers) instead of N replicas")
+    ap.add_argument("--same-device", action="store_true",
+                    help="--sharded only: every process uses cuda:0 and the gloo backend (a functional check on a one-GPU box)")
     ap.add_argument("--mode", default="auto", choices=["walk", "walk_plan_order", "walk_bulk", "auto", "steps", "graph"])
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -524,9 +529,98 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+# --------------------------------------------------------------------------- one broadcast over N GPUs
+def run_sharded(args):
+    """The P ranks spread over the N processes' GPUs.  Strong scaling: the work is one broadcast."""
+    import torch
+    import torch.distributed as dist
+
+    from paper_1603_06809_b200.build import ensure_built
+    ensure_built()
+    from paper_1603_06809_b200 import bcast as B
+    from paper_1603_06809_b200 import workloads as W
+    from paper_1603_06809_b200.sharded import ShardedBroadcast
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = 0 if args.same_device else int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        if args.same_device:
+            dist.init_process_group("gloo")
+        else:
+            dist.init_process_group("nccl", device_id=dev)
+    gather = dist.all_gather_object if world > 1 else (lambda out, obj: out.__setitem__(0, obj))
+    barrier = dist.barrier if world > 1 else (lambda: None)
+    wl = pick_workload(args.workload)
+    P, n = wl.P, wl.nbytes
+    msg_np = W.message_bytes(wl.seed, n)
+    results = {}
+    for name, variant in (("tuned", B.BCAST_TUNED), ("native", B.BCAST_NATIVE)):
+        sb = ShardedBroadcast(P, wl.root, n, variant, rank, world, dev, gather, barrier)
+        for r in sb.mine:
+            sb.local_view(r).fill_(W.poison_byte(r))
+        if sb.owns(wl.root):
+            sb.local_view(wl.root).copy_(torch.from_numpy(msg_np).to(dev))
+        torch.cuda.synchronize()
+        for _ in range(args.warmup):
+            sb.run()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        barrier()
+        e0.record(sb.stream)
+        for _ in range(args.steps):
+            phases = sb.run()
+        e1.record(sb.stream)
+        torch.cuda.synchronize()
+        barrier()
+        ms = max_over_ranks(e0.elapsed_time(e1), world, "cpu" if args.same_device else dev) / args.steps
+        msg = torch.from_numpy(msg_np).to(dev)
+        ok = all(torch.equal(sb.local_view(r), msg) for r in sb.mine)
+        bad = max_over_ranks(0.0 if ok else 1.0, world, "cpu" if args.same_device else dev)
+        if bad:
+            raise SystemExit(f"{name}: a rank buffer differs from the root's message")
+        results[name] = dict(ms=ms, phases=phases, crossing=B.bcast_shard_crossing_bytes(sb.shard),
+                             moved=B.bcast_plan_total_bytes(sb.plan))
+        del sb
+        torch.cuda.empty_cache()
+        barrier()
+    if rank == 0:
+        peak, peak_src = measured_peak()
+        t, nat = results["tuned"], results["native"]
+        value = P * n / (t["ms"] * 1e-3) / 1e9
+        line = {
+            "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": round(t["ms"], 5), "higher_is_better": True, "scaling": "strong",
+            "vs_baseline": None, "dtype": "u8", "data": "synthetic",
+            "config": {"workload": f"{wl.name} tuned (P={P}, root={wl.root}, nbytes={n}, uniform random uint8, seed {wl.seed})",
+                       "variant": "tuned", "exec_mode": "sharded: ranks in contiguous groups over the GPUs, one process per GPU, "
+                       "a barrier after each phase", "phases": t["phases"], "same_device": bool(args.same_device),
+                       "l2": f"rank buffers total {P * n / 1e9:.3f} GB over {world} GPU(s); no flush between iterations",
+                       "nvlink_bytes_per_step": t["crossing"], "bytes_moved_per_step": t["moved"]},
+            "roofline": {"bound": "hbm", "achieved": round(value, 1), "peak": peak * world, "unit": "GB/s",
+                         "frac": round(value / (peak * world), 4), "traffic": None, "kernel": "bcast_walk_kernel",
+                         "peak_source": peak_src + f" x {world} GPUs",
+                         "algorithmic_bytes_are": "DRAM floor of a broadcast: P*nbytes, against the sum of the GPUs' copy rates"},
+            "cpu_baseline": None, "e2e": None, "gpu_launches": args.steps * t["phases"] * world, "clocks": None,
+            "native": {"value": round(P * n / (nat["ms"] * 1e-3) / 1e9, 1), "ms_per_step": round(nat["ms"], 5),
+                       "nvlink_bytes_per_step": nat["crossing"], "bytes_moved_per_step": nat["moved"]},
+            "tuned_over_native": round(nat["ms"] / t["ms"], 4),
+        }
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
 if __name__ == "__main__":
     a = parse_args()
     if a.impl == "reference":
         run_reference(a)
+    elif a.sharded:
+        run_sharded(a)
     else:
         run_ours(a)
