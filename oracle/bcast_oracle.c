@@ -27,6 +27,12 @@
  *     block of 2^i chunks that starts at its own relative rank with the low i bits
  *     cleared.  Third variant (2); power-of-two P only.
  *
+ *   - Section II: for medium messages on a non-power-of-two number of processes MPICH's
+ *     broadcast is aware of the nodes: first a binomial-tree broadcast inside the root's
+ *     node, then the scatter-ring-allgather between the nodes, finally a binomial-tree
+ *     broadcast inside every other node.  Simulated by oracle_bcast_simulate_smp() with
+ *     nodes = blocks of consecutive ranks (see the readings below).
+ *
  * The simulation keeps, for every process, the set of chunks it holds; a message
  * is only formed from what its sender holds (checked before anything is copied).
  * No blocking, fusion or reordering: one memcpy per message, steps in the
@@ -47,6 +53,14 @@
  *   - inside one step, messages are listed by ascending destination rank.
  *   - a "message transfer" in the paper's 56/44 and 90/75 counts is a ring
  *     message; scatter messages are counted separately.
+ *   - node-aware broadcast (Section II names the three phases and nothing else): a node
+ *     is a block of ranks_per_node consecutive ranks (the last one may be smaller); a
+ *     node's leader is its lowest rank; the first broadcast runs down a binomial tree
+ *     rooted at the root over the root's node (relative ranks inside the node, the
+ *     tree of Figs. 1-2 with the whole message on every edge); the scatter-ring runs
+ *     between the leaders, nodes numbered relative to the root's node, with
+ *     scatter_size = ceil(nbytes / number of nodes); the last broadcast runs in every
+ *     other node from its leader, all nodes level by level at the same time.
  *
  * Pinned by tests/test_oracle_pins.py against the worked examples of
  * Figs. 1-5, the printed message counts, closed forms, MPI broadcast
@@ -68,18 +82,22 @@ enum { ORC_OK = 0, ORC_E_ARG = -1, ORC_E_NOMEM = -2, ORC_E_CAP = -3,
 
 /* schedule record: 9 x int64, in this order */
 enum { F_PHASE = 0, F_STEP, F_SRC, F_DST, F_CHUNK, F_NCHUNKS, F_OFFSET, F_LEN, F_DEP, F_NFIELDS };
-enum { PH_SCATTER = 0, PH_RING = 1 };
+enum { PH_SCATTER = 0, PH_RING = 1, PH_NODE_FIRST = 2, PH_NODE_LAST = 3 };   /* 2, 3: node-aware variant only */
 enum { SEND_ONLY = 0, RECV_ONLY = 1 };
 
 typedef struct {
     int P, root;
+    int C;                        /* number of chunks the message is cut into (P, or the number of nodes) */
+    int G;                        /* size of the group that runs the scatter and the ring ...            */
+    const int *member;            /* ... and its processes (absolute ranks) by relative rank, or NULL:
+                                     all P processes, relative rank r = absolute rank (r + root) mod P   */
     uint64_t n, S;
     uint8_t *const *buf;          /* NULL: schedule and counters only */
     int64_t *sched, cap, len;
     uint64_t *bytes_sent, *bytes_recv, *msgs_sent, *msgs_recv;   /* [2][P] */
-    uint8_t *holds;               /* holds[k*P + c]: process k (absolute) holds chunk c (relative) */
+    uint8_t *holds;               /* holds[k*C + c]: process k (absolute) holds chunk c (relative) */
     int *rd_lo, *rd_hi;           /* per process: chunk range read from it in the current step */
-    int64_t *writer;              /* writer[k*P + c]: schedule index of the message that last wrote it, -1 = never */
+    int64_t *writer;              /* writer[k*C + c]: schedule index of the message that last wrote it, -1 = never */
 } sim_t;
 
 static uint64_t umin(uint64_t a, uint64_t b) { return a < b ? a : b; }
@@ -95,8 +113,15 @@ static uint64_t chunk_len(const sim_t *s, int c)
     return umin(s->S, s->n - b);
 }
 
-static int rel_of(const sim_t *s, int k) { return k >= s->root ? k - s->root : k - s->root + s->P; }
-static int abs_of(const sim_t *s, int r) { return (r + s->root) % s->P; }
+/* relative rank r of the group <-> absolute rank */
+static int abs_of(const sim_t *s, int r) { return s->member ? s->member[r] : (r + s->root) % s->P; }
+static int rel_of(const sim_t *s, int k)
+{
+    if (!s->member) return k >= s->root ? k - s->root : k - s->root + s->P;
+    for (int r = 0; r < s->G; r++)
+        if (s->member[r] == k) return r;
+    return -1;
+}
 
 typedef struct { int src, dst, chunk, nchunks; } pending_t;
 
@@ -108,13 +133,13 @@ static int by_dst(const void *a, const void *b)
 /* Deliver the messages of one step: check, record, count, copy. */
 static int deliver_step(sim_t *s, int phase, int step, pending_t *m, int nm)
 {
-    const int P = s->P;
+    const int P = s->P, C = s->C;
     qsort(m, (size_t)nm, sizeof *m, by_dst);
 
     /* a process can only send what has arrived at it in an earlier step */
     for (int a = 0; a < nm; a++)
         for (int c = m[a].chunk; c < m[a].chunk + m[a].nchunks; c++)
-            if (!s->holds[(size_t)m[a].src * P + c]) return ORC_E_NOT_HELD;
+            if (!s->holds[(size_t)m[a].src * C + c]) return ORC_E_NOT_HELD;
     /* all sends of a step see the buffers as they were when the step began: nothing a message
        of this step writes may be read by a message of this step, so that copying the messages
        one after the other equals copying them at once */
@@ -138,7 +163,7 @@ static int deliver_step(sim_t *s, int phase, int step, pending_t *m, int nm)
         rec[F_SRC] = m[a].src; rec[F_DST] = m[a].dst;
         rec[F_CHUNK] = c0;     rec[F_NCHUNKS] = m[a].nchunks;
         rec[F_OFFSET] = (int64_t)off; rec[F_LEN] = (int64_t)len;
-        rec[F_DEP] = s->writer[(size_t)m[a].src * P + c0];
+        rec[F_DEP] = s->writer[(size_t)m[a].src * C + c0];
 
         s->bytes_sent[(size_t)phase * P + m[a].src] += len;
         s->bytes_recv[(size_t)phase * P + m[a].dst] += len;
@@ -152,18 +177,19 @@ static int deliver_step(sim_t *s, int phase, int step, pending_t *m, int nm)
         /* records of this step were appended in the same order as m[] */
         const int64_t idx = s->len + a;
         for (int c = m[a].chunk; c < m[a].chunk + m[a].nchunks; c++) {
-            s->holds[(size_t)m[a].dst * P + c] = 1;
-            s->writer[(size_t)m[a].dst * P + c] = idx;
+            s->holds[(size_t)m[a].dst * C + c] = 1;
+            s->writer[(size_t)m[a].dst * C + c] = idx;
         }
     }
     s->len += nm;
     return ORC_OK;
 }
 
-/* Section III-A, Figs. 1-2: binomial scatter from relative rank 0. */
+/* Section III-A, Figs. 1-2: binomial scatter from relative rank 0 of the group (all P processes,
+   or the node leaders of the node-aware variant). */
 static int scatter_phase(sim_t *s, int L, pending_t *m)
 {
-    const int P = s->P;
+    const int P = s->G;
     for (int t = 0; t < L; t++) {
         const int mask = 1 << (L - 1 - t);
         int nm = 0;
@@ -200,25 +226,25 @@ static int scatter_phase(sim_t *s, int L, pending_t *m)
  */
 static int ring_phase(sim_t *s, int tuned, pending_t *m, int *last_recv, int *last_send)
 {
-    const int P = s->P;
+    const int P = s->G, C = s->C;                        /* processes on the ring; chunks per process set */
     int rc = ORC_OK;
-    uint8_t *owned_after_scatter = malloc((size_t)P * (size_t)P);
+    uint8_t *owned_after_scatter = malloc((size_t)s->P * (size_t)C);
     int *passes = malloc(sizeof(int) * (size_t)P), *arrives = malloc(sizeof(int) * (size_t)P);
     if (!owned_after_scatter || !passes || !arrives) { rc = ORC_E_NOMEM; goto out; }
-    memcpy(owned_after_scatter, s->holds, (size_t)P * (size_t)P);
-    for (int k = 0; k < P; k++) {
-        passes[k] = rel_of(s, k);                        /* step 1: the process's own chunk */
-        if (last_recv) last_recv[k] = 0;
-        if (last_send) last_send[k] = 0;
+    memcpy(owned_after_scatter, s->holds, (size_t)s->P * (size_t)C);
+    for (int q = 0; q < P; q++) {                        /* q: position on the ring = relative rank */
+        passes[q] = q;                                   /* step 1: the process's own chunk */
+        if (last_recv) last_recv[abs_of(s, q)] = 0;
+        if (last_send) last_send[abs_of(s, q)] = 0;
     }
 
     for (int i = 1; i < P; i++) {
         int nm = 0;
-        for (int k = 0; k < P; k++) {
-            const int right = (k + 1) % P;
-            const int chunk = passes[k];
-            arrives[right] = chunk;                      /* due at the right neighbour in this step */
-            if (tuned && owned_after_scatter[(size_t)right * P + chunk]) continue;   /* it has that one: nothing is sent */
+        for (int q = 0; q < P; q++) {
+            const int k = abs_of(s, q), qr = (q + 1) % P, right = abs_of(s, qr);
+            const int chunk = passes[q];
+            arrives[qr] = chunk;                         /* due at the right neighbour in this step */
+            if (tuned && owned_after_scatter[(size_t)right * C + chunk]) continue;   /* it has that one: nothing is sent */
             m[nm].src = k; m[nm].dst = right; m[nm].chunk = chunk; m[nm].nchunks = 1;
             nm++;
             if (last_send) last_send[k] = i;
@@ -226,7 +252,7 @@ static int ring_phase(sim_t *s, int tuned, pending_t *m, int *last_recv, int *la
         }
         rc = deliver_step(s, PH_RING, i - 1, m, nm);
         if (rc) goto out;
-        for (int k = 0; k < P; k++) passes[k] = arrives[k];   /* forward what was due in this step */
+        for (int q = 0; q < P; q++) passes[q] = arrives[q];   /* forward what was due in this step */
     }
 out:
     free(owned_after_scatter); free(passes); free(arrives);
@@ -277,67 +303,147 @@ out:
     return rc;
 }
 
+/* Section II: "an intra-node broadcast ... following a binomial tree".  One step of such broadcasts,
+ * for several disjoint groups at once: in level t of a group of `size` processes (mask m =
+ * 2^(L-1-t), L = ceil(log2 size): the tree of Figs. 1-2) every relative rank r that is a multiple of
+ * 2m and has r + m < size passes the WHOLE message (all C chunks) to relative rank r + m.
+ * groups[g] lists the processes of group g by relative rank; groups with fewer levels than t+1 are
+ * idle.  Returns the number of messages formed (0: no group has a level t), or a negative code. */
+static int tree_bcast_step(sim_t *s, int phase, int t, int ngroups, int *const *groups, const int *sizes, pending_t *m)
+{
+    int nm = 0;
+    for (int g = 0; g < ngroups; g++) {
+        int L = 0;
+        while ((1 << L) < sizes[g]) L++;
+        if (t >= L) continue;
+        const int mask = 1 << (L - 1 - t);
+        for (int r = 0; r + mask < sizes[g]; r += 2 * mask) {
+            m[nm].src = groups[g][r];
+            m[nm].dst = groups[g][r + mask];
+            m[nm].chunk = 0;
+            m[nm].nchunks = s->C;
+            nm++;
+        }
+    }
+    if (nm == 0) return 0;
+    const int rc = deliver_step(s, phase, t, m, nm);
+    return rc ? rc : nm;
+}
+
 /*
  * Simulate one broadcast.
  *   P, root, nbytes   communicator size, root rank, message bytes
  *   tuned             0: native ring (Section III-A), 1: tuned ring (Section IV),
  *                     2: recursive-doubling allgather in place of the ring (Section I; P must be
  *                        a power of two)
+ *   per_node          0: no node awareness (everything above).  >= 1: the node-aware broadcast of
+ *                     Section II with nodes of per_node consecutive ranks: binomial-tree broadcast in
+ *                     the root's node, scatter + (native or tuned) ring between the node leaders with
+ *                     the message cut into as many chunks as there are nodes, binomial-tree
+ *                     broadcast in every other node (tuned = 2 is not defined here)
  *   buf               P host buffers of nbytes each; buf[root] holds the message.  NULL: no data is
  *                     moved, only the schedule and the counters are produced.
  *   sched, cap        room for cap records of 9 int64 (phase, step, src, dst, chunk, nchunks,
  *                     offset, len, dep); *nsched receives the number written
- *   bytes_sent ...    four arrays [2][P] (phase, absolute rank), zeroed here
+ *   bytes_sent ...    four arrays [nphases][P] (phase, absolute rank), zeroed here; nphases is 2
+ *                     without node awareness and 4 with it
  * Returns ORC_OK or a negative ORC_E_* code.
  */
-static int simulate(int P, int root, uint64_t nbytes, int tuned, uint8_t *const *buf,
+static int simulate(int P, int root, uint64_t nbytes, int tuned, int per_node, uint8_t *const *buf,
                     int64_t *sched, int64_t cap, int64_t *nsched,
                     uint64_t *bytes_sent, uint64_t *bytes_recv,
                     uint64_t *msgs_sent, uint64_t *msgs_recv, int *last_recv, int *last_send)
 {
-    if (P < 1 || root < 0 || root >= P || !sched || !nsched || cap < 0 ||
+    if (P < 1 || root < 0 || root >= P || !sched || !nsched || cap < 0 || per_node < 0 ||
         !bytes_sent || !bytes_recv || !msgs_sent || !msgs_recv)
         return ORC_E_ARG;
-    if (tuned < 0 || tuned > 2 || (tuned == 2 && (P & (P - 1)) != 0)) return ORC_E_ARG;
+    if (tuned < 0 || tuned > 2 || (tuned == 2 && ((P & (P - 1)) != 0 || per_node))) return ORC_E_ARG;
 
+    const int nnodes = per_node ? (P + per_node - 1) / per_node : 0;
+    const int C = per_node ? nnodes : P;                      /* chunks: one per process on the ring */
+    const int nphases = per_node ? 4 : 2;
     sim_t s;
     memset(&s, 0, sizeof s);
-    s.P = P; s.root = root; s.n = nbytes;
-    s.S = (nbytes + (uint64_t)P - 1) / (uint64_t)P;          /* scatter_size, Section IV listing */
+    s.P = P; s.root = root; s.n = nbytes; s.C = C; s.G = P; s.member = NULL;
+    s.S = (nbytes + (uint64_t)C - 1) / (uint64_t)C;          /* scatter_size, Section IV listing */
     s.buf = buf; s.sched = sched; s.cap = cap; s.len = 0;
     s.bytes_sent = bytes_sent; s.bytes_recv = bytes_recv; s.msgs_sent = msgs_sent; s.msgs_recv = msgs_recv;
-    memset(bytes_sent, 0, sizeof(uint64_t) * 2 * (size_t)P);
-    memset(bytes_recv, 0, sizeof(uint64_t) * 2 * (size_t)P);
-    memset(msgs_sent, 0, sizeof(uint64_t) * 2 * (size_t)P);
-    memset(msgs_recv, 0, sizeof(uint64_t) * 2 * (size_t)P);
+    memset(bytes_sent, 0, sizeof(uint64_t) * (size_t)nphases * (size_t)P);
+    memset(bytes_recv, 0, sizeof(uint64_t) * (size_t)nphases * (size_t)P);
+    memset(msgs_sent, 0, sizeof(uint64_t) * (size_t)nphases * (size_t)P);
+    memset(msgs_recv, 0, sizeof(uint64_t) * (size_t)nphases * (size_t)P);
 
     int rc = ORC_OK;
     pending_t *m = malloc(sizeof(pending_t) * (size_t)P);
-    s.holds = calloc((size_t)P * (size_t)P, 1);
-    s.writer = malloc(sizeof(int64_t) * (size_t)P * (size_t)P);
+    s.holds = calloc((size_t)P * (size_t)C, 1);
+    s.writer = malloc(sizeof(int64_t) * (size_t)P * (size_t)C);
     s.rd_lo = malloc(sizeof(int) * (size_t)P);
     s.rd_hi = malloc(sizeof(int) * (size_t)P);
-    if (!m || !s.holds || !s.writer || !s.rd_lo || !s.rd_hi) { rc = ORC_E_NOMEM; goto out; }
-    for (size_t x = 0; x < (size_t)P * (size_t)P; x++) s.writer[x] = -1;
-    for (int c = 0; c < P; c++) s.holds[(size_t)root * P + c] = 1;   /* the root has the whole message */
+    int *order = malloc(sizeof(int) * (size_t)P * 2);         /* node-aware: processes by node, leaders */
+    int **groups = malloc(sizeof(int *) * (size_t)(nnodes + 1));
+    int *sizes = malloc(sizeof(int) * (size_t)(nnodes + 1));
+    if (!m || !s.holds || !s.writer || !s.rd_lo || !s.rd_hi || !order || !groups || !sizes) { rc = ORC_E_NOMEM; goto out; }
+    for (size_t x = 0; x < (size_t)P * (size_t)C; x++) s.writer[x] = -1;
+    for (int c = 0; c < C; c++) s.holds[(size_t)root * C + c] = 1;   /* the root has the whole message */
+
+    if (per_node) {
+        /* Section II, first phase: binomial-tree broadcast inside the root's node, rooted at the root */
+        const int root_node = root / per_node;
+        const int first = root_node * per_node, size = (first + per_node <= P ? per_node : P - first);
+        for (int r = 0; r < size; r++) order[r] = first + (root - first + r) % size;    /* relative rank r of the node */
+        groups[0] = order; sizes[0] = size;
+        for (int t = 0;; t++) {
+            rc = tree_bcast_step(&s, PH_NODE_FIRST, t, 1, groups, sizes, m);
+            if (rc < 0) goto out;
+            if (rc == 0) break;
+        }
+        /* second phase: scatter and ring between the node leaders (lowest rank of each node),
+           nodes numbered relative to the root's node */
+        int *leaders = order + P;
+        for (int q = 0; q < nnodes; q++) leaders[q] = ((root_node + q) % nnodes) * per_node;
+        s.G = nnodes; s.member = leaders;
+        /* the leader of the root's node now stands for the root: it holds the whole message */
+        for (int c = 0; c < C; c++)
+            if (!s.holds[(size_t)leaders[0] * C + c]) { rc = ORC_E_NOT_HELD; goto out; }
+    }
 
     int L = 0;
-    while ((1 << L) < P) L++;                                 /* ceil(log2 P) scatter levels */
+    while ((1 << L) < s.G) L++;                               /* ceil(log2) scatter levels */
 
     rc = scatter_phase(&s, L, m);
     if (rc) goto out;
     rc = tuned == 2 ? doubling_phase(&s, m) : ring_phase(&s, tuned, m, last_recv, last_send);
     if (rc) goto out;
 
+    if (per_node) {
+        /* third phase: binomial-tree broadcast inside every other node, from its leader, all nodes at once */
+        const int root_node = root / per_node;
+        int ng = 0;
+        for (int node = 0; node < nnodes; node++) {
+            if (node == root_node) continue;
+            const int first = node * per_node, size = (first + per_node <= P ? per_node : P - first);
+            int *list = order + first;                        /* the node's own stretch of `order` (the root's node is done with it) */
+            for (int r = 0; r < size; r++) list[r] = first + r;
+            groups[ng] = list; sizes[ng] = size; ng++;
+        }
+        for (int t = 0; ng; t++) {
+            rc = tree_bcast_step(&s, PH_NODE_LAST, t, ng, groups, sizes, m);
+            if (rc < 0) goto out;
+            if (rc == 0) break;
+        }
+        rc = ORC_OK;
+    }
+
     /* MPI broadcast semantics (Section III-A): on return every process has the root's message */
-    for (size_t x = 0; x < (size_t)P * (size_t)P; x++)
+    for (size_t x = 0; x < (size_t)P * (size_t)C; x++)
         if (!s.holds[x]) { rc = ORC_E_INCOMPLETE; goto out; }
     if (buf && nbytes)
         for (int k = 0; k < P; k++)
             if (memcmp(buf[k], buf[root], (size_t)nbytes) != 0) { rc = ORC_E_MISMATCH; goto out; }
 out:
+    if (rc > 0) rc = ORC_OK;
     *nsched = s.len;
-    free(m); free(s.holds); free(s.writer); free(s.rd_lo); free(s.rd_hi);
+    free(m); free(s.holds); free(s.writer); free(s.rd_lo); free(s.rd_hi); free(order); free(groups); free(sizes);
     return rc;
 }
 
@@ -346,7 +452,18 @@ int oracle_bcast_simulate(int P, int root, uint64_t nbytes, int tuned, uint8_t *
                           uint64_t *bytes_sent, uint64_t *bytes_recv,
                           uint64_t *msgs_sent, uint64_t *msgs_recv)
 {
-    return simulate(P, root, nbytes, tuned, buf, sched, cap, nsched, bytes_sent, bytes_recv,
+    return simulate(P, root, nbytes, tuned, 0, buf, sched, cap, nsched, bytes_sent, bytes_recv,
+                    msgs_sent, msgs_recv, NULL, NULL);
+}
+
+/* The node-aware broadcast of Section II; counter arrays are [4][P] (phases 0..3, see PH_*). */
+int oracle_bcast_simulate_smp(int P, int root, uint64_t nbytes, int tuned, int ranks_per_node, uint8_t *const *buf,
+                              int64_t *sched, int64_t cap, int64_t *nsched,
+                              uint64_t *bytes_sent, uint64_t *bytes_recv,
+                              uint64_t *msgs_sent, uint64_t *msgs_recv)
+{
+    if (ranks_per_node < 1) return ORC_E_ARG;
+    return simulate(P, root, nbytes, tuned, ranks_per_node, buf, sched, cap, nsched, bytes_sent, bytes_recv,
                     msgs_sent, msgs_recv, NULL, NULL);
 }
 
@@ -372,7 +489,7 @@ int oracle_bcast_step_flag(int P, int *step, int *flag)
     uint64_t *cnt = malloc(sizeof(uint64_t) * 8 * (size_t)P);
     int *last_recv = malloc(sizeof(int) * (size_t)P), *last_send = malloc(sizeof(int) * (size_t)P);
     if (sched && cnt && last_recv && last_send) {
-        rc = simulate(P, 0, (uint64_t)P, 1, NULL, sched, cap, &nsched, cnt, cnt + 2 * P, cnt + 4 * P, cnt + 6 * P,
+        rc = simulate(P, 0, (uint64_t)P, 1, 0, NULL, sched, cap, &nsched, cnt, cnt + 2 * P, cnt + 4 * P, cnt + 6 * P,
                       last_recv, last_send);
         for (int r = 0; !rc && r < P; r++) step_and_flag(P, last_recv[r], last_send[r], &step[r], &flag[r]);
     }

@@ -22,6 +22,7 @@ _LIB = os.path.join(_HERE, "_build", "libbcast_oracle.so")
 
 NATIVE, TUNED, DOUBLING = 0, 1, 2
 SCATTER, RING = 0, 1
+NODE_FIRST, NODE_LAST = 2, 3     # node-aware broadcast only: tree broadcast in the root's node / in the other nodes
 SEND_ONLY, RECV_ONLY = 0, 1
 
 #: column names of the schedule array returned by :func:`simulate`
@@ -55,6 +56,11 @@ def _bind(path: str):
     lib.oracle_bcast_simulate.restype = ctypes.c_int
     lib.oracle_bcast_simulate.argtypes = [
         ctypes.c_int, ctypes.c_int, ctypes.c_uint64, ctypes.c_int, ctypes.POINTER(ctypes.c_void_p),
+        ctypes.POINTER(ctypes.c_int64), ctypes.c_int64, ctypes.POINTER(ctypes.c_int64),
+        u64p, u64p, u64p, u64p]
+    lib.oracle_bcast_simulate_smp.restype = ctypes.c_int
+    lib.oracle_bcast_simulate_smp.argtypes = [
+        ctypes.c_int, ctypes.c_int, ctypes.c_uint64, ctypes.c_int, ctypes.c_int, ctypes.POINTER(ctypes.c_void_p),
         ctypes.POINTER(ctypes.c_int64), ctypes.c_int64, ctypes.POINTER(ctypes.c_int64),
         u64p, u64p, u64p, u64p]
     lib.oracle_bcast_scatter_size.restype = ctypes.c_uint64
@@ -130,13 +136,15 @@ def capacity(P: int) -> int:
 
 
 def simulate(P: int, root: int, nbytes: int, variant: int, message: np.ndarray | None = None,
-             bufs: np.ndarray | None = None) -> OracleResult:
+             bufs: np.ndarray | None = None, ranks_per_node: int = 0) -> OracleResult:
     """Run the simulated broadcast.
 
     ``message``: uint8 array of ``nbytes`` (the root's data) -> per-rank buffers are created here,
     non-root ones filled with a rank-dependent poison.  ``bufs``: a caller-made (P, nbytes) uint8
     array used in place (the caller has put the message into ``bufs[root]``).  Neither: schedule
-    and counters only, no data moved.
+    and counters only, no data moved.  ``ranks_per_node`` >= 1: the node-aware broadcast (tree
+    broadcast in the root's node, scatter-ring between the node leaders, tree broadcast in the
+    other nodes); the counter arrays then have four phases.
     """
     lib = _load()
     if bufs is None and message is not None:
@@ -154,18 +162,26 @@ def simulate(P: int, root: int, nbytes: int, variant: int, message: np.ndarray |
     cap = capacity(P)
     sched = np.zeros((cap, len(FIELDS)), dtype=np.int64)
     nsched = ctypes.c_int64(0)
-    cnt = [np.zeros((2, P), dtype=np.uint64) for _ in range(4)]
+    nphases = 4 if ranks_per_node else 2
+    cnt = [np.zeros((nphases, P), dtype=np.uint64) for _ in range(4)]
     u64p = ctypes.POINTER(ctypes.c_uint64)
     t0 = time.perf_counter()
-    rc = lib.oracle_bcast_simulate(
-        P, root, nbytes, variant, ptrs,
-        sched.ctypes.data_as(ctypes.POINTER(ctypes.c_int64)), cap, ctypes.byref(nsched),
-        *[c.ctypes.data_as(u64p) for c in cnt])
+    if ranks_per_node:
+        rc = lib.oracle_bcast_simulate_smp(
+            P, root, nbytes, variant, ranks_per_node, ptrs,
+            sched.ctypes.data_as(ctypes.POINTER(ctypes.c_int64)), cap, ctypes.byref(nsched),
+            *[c.ctypes.data_as(u64p) for c in cnt])
+    else:
+        rc = lib.oracle_bcast_simulate(
+            P, root, nbytes, variant, ptrs,
+            sched.ctypes.data_as(ctypes.POINTER(ctypes.c_int64)), cap, ctypes.byref(nsched),
+            *[c.ctypes.data_as(u64p) for c in cnt])
     dt = time.perf_counter() - t0
     if rc:
         raise OracleError(rc)
+    nchunks = -(-P // ranks_per_node) if ranks_per_node else P
     return OracleResult(P=P, root=root, nbytes=nbytes, variant=variant,
-                        scatter_size=scatter_size(P, nbytes),
+                        scatter_size=scatter_size(nchunks, nbytes),
                         schedule=sched[: nsched.value].copy(),
                         bytes_sent=cnt[0], bytes_recv=cnt[1], msgs_sent=cnt[2], msgs_recv=cnt[3],
                         bufs=bufs, seconds=dt)

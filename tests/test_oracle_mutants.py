@@ -14,25 +14,25 @@ SRC = os.path.join(ROOT, "oracle", "bcast_oracle.c")
 
 # (name, text in the source, replacement)
 MUTANTS = [
-    ("scatter_size_rounds_down", "s.S = (nbytes + (uint64_t)P - 1) / (uint64_t)P;", "s.S = P ? nbytes / (uint64_t)P : 0;"),
-    ("scatter_levels_in_reverse", "const int mask = 1 << (L - 1 - t);", "const int mask = 1 << t;"),
+    ("scatter_size_rounds_down", "s.S = (nbytes + (uint64_t)C - 1) / (uint64_t)C;", "s.S = C ? nbytes / (uint64_t)C : 0;"),
+    ("scatter_levels_in_reverse", "const int mask = 1 << (L - 1 - t);\n        int nm = 0;", "const int mask = 1 << t;\n        int nm = 0;"),
     ("child_keeps_only_its_own_chunk", "m[nm].nchunks = hi - (r + mask);", "m[nm].nchunks = 1;"),
-    ("tuned_ring_skips_nothing", "if (tuned && owned_after_scatter[(size_t)right * P + chunk]) continue;",
-     "if (0 && tuned && owned_after_scatter[(size_t)right * P + chunk]) continue;"),
-    ("tuned_ring_skips_by_what_the_sender_owned", "if (tuned && owned_after_scatter[(size_t)right * P + chunk]) continue;",
-     "if (tuned && owned_after_scatter[(size_t)k * P + chunk]) continue;"),
-    ("skipped_transfer_stalls_the_rotation", "arrives[right] = chunk;                      /* due",
-     "arrives[right] = (tuned && owned_after_scatter[(size_t)right * P + chunk]) ? passes[right] : chunk;   /* due"),
-    ("ring_turns_the_other_way", "const int right = (k + 1) % P;\n            const int chunk = passes[k];",
-     "const int right = (k + P - 1) % P;\n            const int chunk = passes[k];"),
-    ("ring_chunk_by_absolute_rank", "passes[k] = rel_of(s, k);", "passes[k] = k;"),
-    ("ring_keeps_passing_the_own_chunk", "for (int k = 0; k < P; k++) passes[k] = arrives[k];", "(void)arrives;"),
+    ("tuned_ring_skips_nothing", "if (tuned && owned_after_scatter[(size_t)right * C + chunk]) continue;",
+     "if (0 && tuned && owned_after_scatter[(size_t)right * C + chunk]) continue;"),
+    ("tuned_ring_skips_by_what_the_sender_owned", "if (tuned && owned_after_scatter[(size_t)right * C + chunk]) continue;",
+     "if (tuned && owned_after_scatter[(size_t)k * C + chunk]) continue;"),
+    ("skipped_transfer_stalls_the_rotation", "arrives[qr] = chunk;                         /* due",
+     "arrives[qr] = (tuned && owned_after_scatter[(size_t)right * C + chunk]) ? passes[qr] : chunk;   /* due"),
+    ("ring_turns_the_other_way", "const int k = abs_of(s, q), qr = (q + 1) % P, right = abs_of(s, qr);",
+     "const int k = abs_of(s, q), qr = (q + P - 1) % P, right = abs_of(s, qr);"),
+    ("ring_chunk_by_absolute_rank", "passes[q] = q;                                   /* step 1", "passes[q] = abs_of(s, q);                        /* step 1"),
+    ("ring_keeps_passing_the_own_chunk", "for (int q = 0; q < P; q++) passes[q] = arrives[q];", "(void)arrives;"),
     ("send_only_and_recv_only_swapped", "*flag = last_send <= last_recv ? RECV_ONLY : SEND_ONLY;",
      "*flag = last_send <= last_recv ? SEND_ONLY : RECV_ONLY;"),
     ("step_from_the_receiving_side_only", "const int two_sided_until = last_recv < last_send ? last_recv : last_send;",
      "const int two_sided_until = last_recv; (void)last_send;"),
     ("two_sided_phase_one_step_long", "*step = P - two_sided_until;", "*step = P - two_sided_until - 1;"),
-    ("dep_forgotten", "rec[F_DEP] = s->writer[(size_t)m[a].src * P + c0];", "rec[F_DEP] = -1;"),
+    ("dep_forgotten", "rec[F_DEP] = s->writer[(size_t)m[a].src * C + c0];", "rec[F_DEP] = -1;"),
     ("messages_sorted_by_sender", "return ((const pending_t *)a)->dst - ((const pending_t *)b)->dst;",
      "return ((const pending_t *)b)->src - ((const pending_t *)a)->src;"),
     ("sent_bytes_booked_to_receiver", "s->bytes_sent[(size_t)phase * P + m[a].src] += len;",
@@ -42,6 +42,14 @@ MUTANTS = [
     ("doubling_sends_one_chunk_of_the_block", "m[nm].nchunks = mask;", "m[nm].nchunks = 1;"),
     ("doubling_partner_by_relative_rank", "wants_from[k] = abs_of(s, partner);", "wants_from[k] = partner;"),
     ("doubling_block_of_the_wrong_size", "const int my_block = (r >> i) << i;", "const int my_block = (r >> (i + 1)) << (i + 1);"),
+    # ---- the node-aware broadcast (Section II)
+    ("node_tree_passes_one_chunk_only", "m[nm].nchunks = s->C;", "m[nm].nchunks = 1;"),
+    ("node_tree_levels_in_reverse", "const int mask = 1 << (L - 1 - t);\n        for (int r = 0; r + mask < sizes[g]; r += 2 * mask) {",
+     "const int mask = 1 << t;\n        for (int r = 0; r + mask < sizes[g]; r += 2 * mask) {"),
+    ("first_tree_rooted_at_the_node_leader", "order[r] = first + (root - first + r) % size;", "order[r] = first + r;"),
+    ("leaders_not_relative_to_the_root_node", "leaders[q] = ((root_node + q) % nnodes) * per_node;", "leaders[q] = q * per_node;"),
+    ("last_trees_also_in_the_root_node", "if (node == root_node) continue;", "if (0 && node == root_node) continue;"),
+    ("node_chunks_as_many_as_processes", "const int C = per_node ? nnodes : P;", "const int C = P; (void)nnodes;"),
     ("offset_not_clipped", "static uint64_t chunk_begin(const sim_t *s, int c) { return umin((uint64_t)c * s->S, s->n); }",
      "static uint64_t chunk_begin(const sim_t *s, int c) { return (uint64_t)c * s->S; }"),
 ]
@@ -72,6 +80,10 @@ def schedule_level_pins(oracle):
     for case in ((4, 1, 3), (16, 15, 65521), (64, 17, (16 << 20) + 13)):
         yield lambda case=case: pins.test_doubling_byte_budget_and_semantics(oracle, *case, with_data=False)
     yield lambda: pins.test_doubling_root_rotation_and_validity(oracle)
+    for case in pins.SMP_CASES:
+        yield lambda case=case: pins.test_node_aware_structure(oracle, *case)
+    yield lambda: pins.test_node_aware_degenerate_cases(oracle)
+    yield lambda: pins.test_node_aware_leader_ring_is_the_plain_ring_of_the_nodes(oracle)
 
 
 def test_the_unbroken_oracle_passes_the_same_pins(oracle):

@@ -438,3 +438,125 @@ def test_doubling_root_rotation_and_validity(oracle):
         assert keys == sorted(keys) and len(set(keys)) == len(keys)
         for x, row in enumerate(res.schedule):
             assert -1 <= int(row[8]) < x
+
+
+# ----------------------------------------------------------------------------- node-aware broadcast
+# Section II: tree broadcast in the root's node, scatter-ring between the nodes, tree broadcast in the
+# other nodes.  The paper prints no worked example for it, so the pins are structural: the trees
+# against recursive halving (the tree of Figs. 1-2, pinned above, carrying the whole message), the
+# part between the nodes against the plain schedule of as many processes as there are nodes (pinned
+# above by Figs. 1-5), explicit holder sets, byte budgets and MPI semantics.
+NODE_FIRST, NODE_LAST = 2, 3
+SMP_CASES = [(12, 5, 1000, 4), (12, 0, 4096, 3), (10, 7, 777, 3), (24, 13, 24 * 100 + 1, 6), (9, 2, 64, 4), (16, 15, 5000, 4),
+             (7, 3, 50, 2), (33, 20, 33 * 31, 8), (6, 5, 3, 5)]
+
+
+def tree_by_halving(members):
+    """(level, src, dst) of a binomial broadcast over `members` (relative rank order), by recursive halving."""
+    size = len(members)
+    if size <= 1:
+        return set()
+    L = (size - 1).bit_length()
+    depth = {1 << b: b for b in range(L + 1)}
+    edges = []
+    halving_tree(0, size, edges, depth, L)
+    return {(level, members[src], members[dst]) for level, src, dst, _ in edges}
+
+
+@pytest.mark.parametrize("P,root,n,c", SMP_CASES)
+def test_node_aware_structure(oracle, P, root, n, c):
+    nodes = [list(range(f, min(f + c, P))) for f in range(0, P, c)]
+    k = len(nodes)
+    root_node = root // c
+    leaders = [nd[0] for nd in nodes]
+    S = -(-n // k)
+    for variant in (NATIVE, TUNED):
+        res = oracle.simulate(P, root, n, variant, ranks_per_node=c)
+        assert res.scatter_size == S
+        sch = res.schedule
+        phase = sch[:, 0]
+        # the phases come in the order of Section II: first tree, scatter, ring, last trees
+        order = [int(p) for i, p in enumerate(phase) if i == 0 or p != phase[i - 1]]
+        assert order == [p for p in (NODE_FIRST, SCATTER, RING, NODE_LAST) if (phase == p).any()]
+        # first tree: over the root's node, rooted at the root, the whole message on every edge
+        rn = nodes[root_node]
+        members = [rn[(rn.index(root) + r) % len(rn)] for r in range(len(rn))]
+        first = sch[phase == NODE_FIRST]
+        assert {(int(r[1]), int(r[2]), int(r[3])) for r in first} == tree_by_halving(members)
+        assert (first[:, 4] == 0).all() and (first[:, 5] == k).all() and (first[:, 6] == 0).all() and (first[:, 7] == n).all()
+        # last trees: in every other node from its lowest rank, all nodes level by level together
+        want = set()
+        for i, nd in enumerate(nodes):
+            if i != root_node:
+                want |= tree_by_halving(nd)
+        last = sch[phase == NODE_LAST]
+        assert {(int(r[1]), int(r[2]), int(r[3])) for r in last} == want
+        assert (last[:, 7] == n).all() and (last[:, 5] == k).all()
+        # between the nodes only leaders talk
+        inter = sch[(phase == SCATTER) | (phase == RING)]
+        assert set(inter[:, 2].tolist()) | set(inter[:, 3].tolist()) <= set(leaders)
+        # holder sets: nothing is sent that has not arrived; in the end everybody holds every chunk
+        holds = [set() for _ in range(P)]
+        holds[root] = set(range(k))
+        i = 0
+        while i < len(sch):
+            j = i
+            while j < len(sch) and (sch[j, 0], sch[j, 1]) == (sch[i, 0], sch[i, 1]):
+                j += 1
+            for row in sch[i:j]:
+                assert set(range(int(row[4]), int(row[4] + row[5]))) <= holds[int(row[2])]
+            for row in sch[i:j]:
+                holds[int(row[3])] |= set(range(int(row[4]), int(row[4] + row[5])))
+            i = j
+        assert all(h == set(range(k)) for h in holds)
+        # byte budget
+        assert int(first[:, 7].sum()) == (len(rn) - 1) * n
+        assert int(last[:, 7].sum()) == sum(len(nd) - 1 for i, nd in enumerate(nodes) if i != root_node) * n
+        if variant == TUNED:
+            assert int(inter[:, 7].sum()) == (k - 1) * n             # every other leader receives the message once
+            assert int(sch[:, 7].sum()) == (P - 1) * n               # and every process but the root, in total
+            per_rank = np.bincount(sch[:, 3], weights=sch[:, 7], minlength=P)
+            assert all(int(per_rank[r]) == (0 if r == root else n) for r in range(P))
+        for ph in range(4):
+            rows = sch[phase == ph]
+            assert np.array_equal(res.bytes_recv[ph], np.bincount(rows[:, 3], weights=rows[:, 7], minlength=P).astype(np.uint64))
+            assert np.array_equal(res.msgs_sent[ph], np.bincount(rows[:, 2], minlength=P).astype(np.uint64))
+    # data
+    msg = np.random.default_rng(P * 1000 + c).integers(0, 256, size=n, dtype=np.uint8)
+    res = oracle.simulate(P, root, n, TUNED, message=msg, ranks_per_node=c)
+    assert (res.bufs == msg[None, :]).all()
+
+
+def test_node_aware_leader_ring_is_the_plain_ring_of_the_nodes(oracle):
+    """With P = c * k, what happens between the nodes is the plain scatter-ring of k processes
+    (the one Figs. 1-5 pin), process j standing for the leader of node j."""
+    for c, k, root, n in [(4, 8, 13, 8 * 512 + 3), (3, 10, 29, 10 * 100), (2, 12, 0, 4099), (5, 3, 7, 100)]:
+        P = c * k
+        for variant in (NATIVE, TUNED):
+            smp = oracle.simulate(P, root, n, variant, ranks_per_node=c)
+            plain = oracle.simulate(k, root // c, n, variant)
+            inter = smp.schedule[(smp.schedule[:, 0] == SCATTER) | (smp.schedule[:, 0] == RING)]
+            assert len(inter) == len(plain.schedule)
+            a = inter.copy()
+            a[:, 2] //= c
+            a[:, 3] //= c
+            assert (inter[:, 2] % c == 0).all() and (inter[:, 3] % c == 0).all()
+            assert np.array_equal(a[:, :8], plain.schedule[:, :8])          # all but `dep`
+
+
+def test_node_aware_degenerate_cases(oracle):
+    """One process per node: nothing but the plain scatter-ring.  One node: nothing but a tree
+    broadcast, ceil(log2 P) steps, P - 1 messages of the whole message."""
+    for P, root, n in [(8, 3, 1000), (10, 0, 77), (5, 4, 5)]:
+        for variant in (NATIVE, TUNED):
+            a = oracle.simulate(P, root, n, variant, ranks_per_node=1)
+            b = oracle.simulate(P, root, n, variant)
+            assert np.array_equal(a.schedule, b.schedule)
+        one = oracle.simulate(P, root, n, TUNED, ranks_per_node=P + 3)
+        assert (one.schedule[:, 0] == NODE_FIRST).all() and len(one.schedule) == P - 1
+        assert int(one.schedule[:, 1].max()) + 1 == (P - 1).bit_length()
+        assert (one.schedule[:, 7] == n).all() and one.scatter_size == n
+        members = [(root + r) % P for r in range(P)]
+        assert {(int(r[1]), int(r[2]), int(r[3])) for r in one.schedule} == tree_by_halving(members)
+    with pytest.raises(oracle.OracleError):
+        oracle.simulate(8, 0, 100, 2, ranks_per_node=2)              # no recursive doubling between nodes here
