@@ -58,8 +58,10 @@ extern "C" {
    number of processes (named in Section I; the standard hypercube exchange): log2 P exchanges, in
    exchange i relative rank r swaps with r xor 2^i the block of 2^i chunks around each of them. */
 enum { BCAST_NATIVE = 0, BCAST_TUNED = 1, BCAST_DOUBLING = 2 };
-/* phase of a message; BCAST_PHASE_RING is the allgather phase (ring steps, or doubling exchanges) */
-enum { BCAST_PHASE_SCATTER = 0, BCAST_PHASE_RING = 1 };
+/* phase of a message; BCAST_PHASE_RING is the allgather phase (ring steps, or doubling exchanges).
+   The node-aware broadcast (bcast_plan_smp) has two more: the tree broadcast inside the root's node,
+   which comes before the scatter, and the tree broadcasts inside the other nodes, which come last. */
+enum { BCAST_PHASE_SCATTER = 0, BCAST_PHASE_RING = 1, BCAST_PHASE_NODE_FIRST = 2, BCAST_PHASE_NODE_LAST = 3 };
 
 enum {
     BCAST_OK = 0,
@@ -141,6 +143,29 @@ typedef struct bcast_plan bcast_plan_t; /* opaque; created and freed by the libr
  */
 int bcast_plan(int P, int root, uint64_t nbytes, int variant, bcast_plan_t **out);
 
+/*
+ * bcast_plan_smp -- the node-aware broadcast that MPICH uses for medium messages on a
+ * non-power-of-two number of processes (Section II): a binomial-tree broadcast inside the root's
+ * node, the scatter-ring-allgather between the nodes, a binomial-tree broadcast inside every other
+ * node.  The paper names the three phases and no more; the readings taken here:
+ *   - a node is a block of ranks_per_node consecutive absolute ranks (the last one may be smaller);
+ *     its leader is its lowest rank;
+ *   - first phase (BCAST_PHASE_NODE_FIRST): the binomial tree of Figs. 1-2 over the root's node,
+ *     rooted at the root (relative ranks inside the node), the whole message on every edge;
+ *   - second phase (BCAST_PHASE_SCATTER, BCAST_PHASE_RING): scatter and native or tuned ring between
+ *     the node leaders, nodes numbered relative to the root's node; the message is cut into as many
+ *     chunks as there are nodes, scatter_size = ceil(nbytes / nodes);
+ *   - third phase (BCAST_PHASE_NODE_LAST): in every other node the same kind of tree from the
+ *     leader, all nodes level by level at the same time (a step holds one level of every node).
+ *   variant         BCAST_NATIVE or BCAST_TUNED: the ring between the leaders
+ *   ranks_per_node  >= 1; 1 gives the schedule of bcast_plan(), >= P a single tree broadcast
+ * Messages are ordered by (NODE_FIRST steps, SCATTER steps, RING steps, NODE_LAST steps), inside a
+ * step by dst_rank; `chunk` counts chunks of scatter_size bytes, relative to the root's node; `dep`
+ * of a whole-message send names the message that last wrote the first chunk into its source.
+ * All executors run such a plan like any other.  Errors: as bcast_plan.
+ */
+int bcast_plan_smp(int P, int root, uint64_t nbytes, int variant, int ranks_per_node, bcast_plan_t **out);
+
 /* Release a plan and the device tables it cached (the device it was executed on must still be
    usable).  NULL is ignored. */
 void bcast_plan_free(bcast_plan_t *plan);
@@ -150,10 +175,13 @@ void bcast_plan_free(bcast_plan_t *plan);
 int32_t bcast_plan_num_ranks(const bcast_plan_t *plan);          /* P                               */
 int32_t bcast_plan_root(const bcast_plan_t *plan);
 int32_t bcast_plan_variant(const bcast_plan_t *plan);
+int32_t bcast_plan_ranks_per_node(const bcast_plan_t *plan);     /* 0 unless made by bcast_plan_smp     */
+int32_t bcast_plan_num_chunks(const bcast_plan_t *plan);         /* P, or the number of nodes           */
 uint64_t bcast_plan_nbytes(const bcast_plan_t *plan);
-uint64_t bcast_plan_scatter_size(const bcast_plan_t *plan);      /* S = ceil(nbytes / P) (Section IV listing) */
+uint64_t bcast_plan_scatter_size(const bcast_plan_t *plan);      /* S = ceil(nbytes / num_chunks) (Section IV listing) */
 int64_t bcast_plan_num_xfers(const bcast_plan_t *plan);          /* number of messages               */
-int32_t bcast_plan_num_steps(const bcast_plan_t *plan);          /* L + (P-1) (doubling: 2L); 0 for P = 1 */
+int32_t bcast_plan_num_steps(const bcast_plan_t *plan);          /* L + (P-1) (doubling: 2L); 0 for P = 1;
+                                                                    node-aware: tree levels + L + (nodes-1) + tree levels */
 const bcast_xfer_t *bcast_plan_xfers(const bcast_plan_t *plan);  /* [num_xfers], canonical order      */
 const int64_t *bcast_plan_step_begin(const bcast_plan_t *plan);  /* [num_steps+1]: messages of step s
                                                                     are [step_begin[s], step_begin[s+1]) */

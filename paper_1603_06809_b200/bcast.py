@@ -20,7 +20,7 @@ _lib = ctypes.CDLL(_LIB_PATH)
 
 BCAST_MAX_RANKS = 1024
 BCAST_NATIVE, BCAST_TUNED, BCAST_DOUBLING = 0, 1, 2
-BCAST_PHASE_SCATTER, BCAST_PHASE_RING = 0, 1
+BCAST_PHASE_SCATTER, BCAST_PHASE_RING, BCAST_PHASE_NODE_FIRST, BCAST_PHASE_NODE_LAST = 0, 1, 2, 3
 BCAST_OK, BCAST_ERR_INVAL, BCAST_ERR_NOMEM, BCAST_ERR_CUDA, BCAST_ERR_CAPACITY, BCAST_ERR_TIMEOUT = 0, -1, -2, -3, -4, -5
 BCAST_STATIC_SCRATCH_BYTES = 2 << 20
 BCAST_EXEC_WALK, BCAST_EXEC_STEPS, BCAST_EXEC_GRAPH, BCAST_EXEC_WALK_PLAN_ORDER = 0, 1, 2, 3
@@ -34,7 +34,8 @@ assert XFER_DTYPE.itemsize == 48
 
 #: every symbol ``include/bcast.h`` declares
 SYMBOLS = (
-    "bcast_plan", "bcast_plan_free", "bcast_plan_num_ranks", "bcast_plan_root", "bcast_plan_variant",
+    "bcast_plan", "bcast_plan_smp", "bcast_plan_free", "bcast_plan_num_ranks", "bcast_plan_root", "bcast_plan_variant",
+    "bcast_plan_ranks_per_node", "bcast_plan_num_chunks",
     "bcast_plan_nbytes", "bcast_plan_scatter_size", "bcast_plan_num_xfers", "bcast_plan_num_steps",
     "bcast_plan_xfers", "bcast_plan_step_begin", "bcast_plan_bytes_sent", "bcast_plan_bytes_recv",
     "bcast_plan_msgs_sent", "bcast_plan_msgs_recv", "bcast_plan_total_bytes", "bcast_plan_walk_order",
@@ -50,6 +51,8 @@ _vp, _i, _i32, _i64, _u64 = ctypes.c_void_p, ctypes.c_int, ctypes.c_int32, ctype
 _vpp = ctypes.POINTER(ctypes.c_void_p)
 _sig = {
     "bcast_plan": (_i, [_i, _i, _u64, _i, _vpp]),
+    "bcast_plan_smp": (_i, [_i, _i, _u64, _i, _i, _vpp]),
+    "bcast_plan_ranks_per_node": (_i32, [_vp]), "bcast_plan_num_chunks": (_i32, [_vp]),
     "bcast_plan_free": (None, [_vp]),
     "bcast_plan_num_ranks": (_i32, [_vp]), "bcast_plan_root": (_i32, [_vp]), "bcast_plan_variant": (_i32, [_vp]),
     "bcast_plan_nbytes": (_u64, [_vp]), "bcast_plan_scatter_size": (_u64, [_vp]),
@@ -136,6 +139,12 @@ def bcast_plan(P: int, root: int, nbytes: int, variant: int) -> Plan:
     return Plan(out.value)
 
 
+def bcast_plan_smp(P: int, root: int, nbytes: int, variant: int, ranks_per_node: int) -> Plan:
+    out = ctypes.c_void_p(None)
+    _check(_lib.bcast_plan_smp(P, root, nbytes, variant, ranks_per_node, ctypes.byref(out)), "bcast_plan_smp")
+    return Plan(out.value)
+
+
 def bcast_plan_free(plan: Plan) -> None:
     plan.free()
 
@@ -143,6 +152,8 @@ def bcast_plan_free(plan: Plan) -> None:
 def bcast_plan_num_ranks(plan: Plan) -> int: return _lib.bcast_plan_num_ranks(plan.handle)
 def bcast_plan_root(plan: Plan) -> int: return _lib.bcast_plan_root(plan.handle)
 def bcast_plan_variant(plan: Plan) -> int: return _lib.bcast_plan_variant(plan.handle)
+def bcast_plan_ranks_per_node(plan: Plan) -> int: return _lib.bcast_plan_ranks_per_node(plan.handle)
+def bcast_plan_num_chunks(plan: Plan) -> int: return _lib.bcast_plan_num_chunks(plan.handle)
 def bcast_plan_nbytes(plan: Plan) -> int: return _lib.bcast_plan_nbytes(plan.handle)
 def bcast_plan_scatter_size(plan: Plan) -> int: return _lib.bcast_plan_scatter_size(plan.handle)
 def bcast_plan_num_xfers(plan: Plan) -> int: return _lib.bcast_plan_num_xfers(plan.handle)

@@ -60,10 +60,10 @@ class RankBuffers:
         return out
 
 
-def run_broadcast(P, root, nbytes, variant, mode, message, shift=0, repeats=1):
+def run_broadcast(P, root, nbytes, variant, mode, message, shift=0, repeats=1, ranks_per_node=0):
     """Plan + execute through the C ABI on cuda:0; returns (plan, RankBuffers) after a sync."""
     bufs = RankBuffers(P, root, nbytes, message, shift=shift)
-    plan = B.bcast_plan(P, root, nbytes, variant)
+    plan = B.bcast_plan_smp(P, root, nbytes, variant, ranks_per_node) if ranks_per_node else B.bcast_plan(P, root, nbytes, variant)
     stream = torch.cuda.current_stream()
     for rep in range(repeats):
         if rep:

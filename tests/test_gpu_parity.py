@@ -308,3 +308,31 @@ def test_exec_rejects_bad_buffers():
     B.bcast_exec(good, plan)
     torch.cuda.synchronize()
     assert bufs.all_equal_message() and bufs.guards_intact()
+
+
+# ---- the node-aware broadcast (Section II) through every executor, and its bytes counted on the device
+SMP_WORKLOADS = [(W.Workload("smp_p12", 12, 5, 256 * 1024 + 5, 51), 4), (W.Workload("smp_p24", 24, 13, 24 * 40961, 52), 6),
+                 (W.Workload("smp_p129", 129, 0, 524287, 53), 24), (W.Workload("smp_p100", 100, 63, (8 << 20) + 1, 54), 8),
+                 (W.Workload("smp_one_node", 9, 2, 70001, 55), 16), (W.Workload("smp_tiny", 33, 20, 700, 56), 8)]
+
+
+@pytest.mark.parametrize("mode", MODES, ids=MODE_IDS)
+@pytest.mark.parametrize("variant", VARIANTS, ids=VARIANT_IDS)
+@pytest.mark.parametrize("wl,c", SMP_WORKLOADS, ids=lambda x: x.name if hasattr(x, "name") else f"c{x}")
+def test_node_aware_broadcast(oracle, wl, c, variant, mode):
+    msg = W.message_bytes(wl.seed, wl.nbytes)
+    plan, bufs = run_broadcast(wl.P, wl.root, wl.nbytes, variant, mode, msg, ranks_per_node=c)
+    B.bcast_exec_status(plan)
+    ref = oracle.simulate(wl.P, wl.root, wl.nbytes, variant, message=msg, ranks_per_node=c)
+    assert np.array_equal(bufs.to_host(), ref.bufs)
+    assert bufs.guards_intact()
+    x = B.bcast_plan_xfers(plan)
+    assert np.array_equal(x["len"].astype(np.int64), ref.col("len"))
+    assert np.array_equal(x["dep"], ref.col("dep"))
+    if mode in (B.BCAST_EXEC_WALK, B.BCAST_EXEC_WALK_BULK, B.BCAST_EXEC_STEPS):
+        bufs.reset()
+        counts = torch.zeros(len(x), dtype=torch.int64, device="cuda:0")
+        B.bcast_exec_traced(bufs.pointers(), plan, torch.cuda.current_stream(), mode, counts)
+        torch.cuda.synchronize()
+        assert np.array_equal(counts.cpu().numpy(), ref.col("len"))       # every message performed in full, once
+        assert bufs.all_equal_message()

@@ -91,3 +91,21 @@ def test_shard_exec_rejects_misplaced_and_bad_arguments():
     B.bcast_shard_exec(shard, good, [0, 0], [st, st])
     torch.cuda.synchronize()
     assert bufs.all_equal_message() and bufs.guards_intact()
+
+
+def test_node_aware_plan_over_partitions(oracle):
+    # nodes of the plan and GPUs of the partition are independent groupings of the ranks
+    wl = W.Workload("shard_smp", 24, 13, 24 * 40961, 29)
+    msg = W.message_bytes(wl.seed, wl.nbytes)
+    for variant in (B.BCAST_NATIVE, B.BCAST_TUNED):
+        bufs = RankBuffers(wl.P, wl.root, wl.nbytes, msg)
+        plan = B.bcast_plan_smp(wl.P, wl.root, wl.nbytes, variant, 6)
+        shard = B.bcast_shard_create(plan, 4)
+        counts = torch.zeros(B.bcast_plan_num_xfers(plan), dtype=torch.int64, device="cuda:0")
+        streams = [torch.cuda.Stream() for _ in range(4)]
+        torch.cuda.synchronize()
+        B.bcast_shard_exec(shard, bufs.pointers(), [0] * 4, streams, counts)
+        torch.cuda.synchronize()
+        ref = oracle.simulate(wl.P, wl.root, wl.nbytes, variant, message=msg, ranks_per_node=6)
+        assert np.array_equal(bufs.to_host(), ref.bufs) and bufs.guards_intact()
+        assert np.array_equal(counts.cpu().numpy(), ref.col("len"))

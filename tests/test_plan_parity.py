@@ -59,7 +59,7 @@ def test_library_exports_every_declared_symbol():
 def test_binding_constants_match_header():
     header = open(os.path.join(ROOT, "include", "bcast.h")).read()
     pairs = dict(re.findall(r"\b(BCAST_[A-Z_]+)\s*=\s*(-?\d+)", header))
-    assert len(pairs) == 17
+    assert len(pairs) == 19
     for name, value in pairs.items():
         assert getattr(B, name) == int(value), name
     assert B.BCAST_MAX_RANKS == int(re.search(r"#define BCAST_MAX_RANKS (\d+)", header).group(1))
@@ -138,7 +138,8 @@ def test_plan_argument_errors():
     assert not B._lib.bcast_plan_bytes_sent(None, 0)
     B._lib.bcast_plan_free(None)
     plan = B.bcast_plan(4, 0, 10, 1)
-    assert not B._lib.bcast_plan_bytes_sent(plan.handle, 2)
+    assert not B._lib.bcast_plan_bytes_sent(plan.handle, 4) and not B._lib.bcast_plan_bytes_sent(plan.handle, -1)
+    assert not B.bcast_plan_bytes_sent(plan, B.BCAST_PHASE_NODE_LAST).any()     # phases of the node-aware broadcast: unused here
     assert B.bcast_strerror(B.BCAST_ERR_INVAL) == "invalid argument" and B.bcast_strerror(0) == "success"
 
 
@@ -251,3 +252,52 @@ def test_plan_equals_oracle_random_shapes(oracle):
         variants = [B.BCAST_NATIVE, B.BCAST_TUNED] + ([B.BCAST_DOUBLING] if P & (P - 1) == 0 else [])
         assert_plan_equals_oracle(oracle, P, root, n, data.draw(st.sampled_from(variants)))
     check()
+
+
+# ---- the node-aware broadcast (Section II): planner (closed form per group) == oracle (simulation)
+SMP_SHAPES = [(12, 5, 1000, 4), (12, 0, 4096, 3), (10, 7, 777, 3), (24, 13, 24 * 100 + 1, 6), (9, 2, 64, 4), (16, 15, 5000, 4),
+              (7, 3, 50, 2), (33, 20, 33 * 31, 8), (6, 5, 3, 5), (100, 63, 1 << 20, 8), (129, 0, 524287, 24), (64, 17, (1 << 20) + 13, 64),
+              (8, 3, 100, 1), (5, 4, 0, 2), (1, 0, 10, 4)]
+
+
+@pytest.mark.parametrize("variant", [B.BCAST_NATIVE, B.BCAST_TUNED], ids=["native", "tuned"])
+@pytest.mark.parametrize("P,root,n,c", SMP_SHAPES)
+def test_node_aware_plan_equals_oracle(oracle, P, root, n, c, variant):
+    plan = B.bcast_plan_smp(P, root, n, variant, c)
+    ref = oracle.simulate(P, root, n, variant, ranks_per_node=c)
+    mine = plan_matrix(plan)
+    assert mine.shape == ref.schedule.shape
+    assert (mine == ref.schedule).all()                       # every field, `dep` included
+    assert B.bcast_plan_scatter_size(plan) == ref.scatter_size
+    assert B.bcast_plan_ranks_per_node(plan) == c and B.bcast_plan_num_chunks(plan) == -(-P // c)
+    for ph in range(4):
+        assert (B.bcast_plan_bytes_sent(plan, ph) == ref.bytes_sent[ph]).all()
+        assert (B.bcast_plan_bytes_recv(plan, ph) == ref.bytes_recv[ph]).all()
+        assert (B.bcast_plan_msgs_sent(plan, ph) == ref.msgs_sent[ph]).all()
+        assert (B.bcast_plan_msgs_recv(plan, ph) == ref.msgs_recv[ph]).all()
+    # CSR over steps: every step holds the messages of one (phase, step)
+    sb = B.bcast_plan_step_begin(plan)
+    assert sb[0] == 0 and sb[-1] == len(mine) and (np.diff(sb) >= 0).all()
+    seen = []
+    for s in range(len(sb) - 1):
+        rows = mine[sb[s]:sb[s + 1]]
+        if len(rows):
+            assert len({(int(r[0]), int(r[1])) for r in rows}) == 1
+            seen.append((int(rows[0, 0]), int(rows[0, 1])))
+    assert seen == sorted(set(seen), key=lambda ps: ({2: 0, 0: 1, 1: 2, 3: 3}[ps[0]], ps[1]))
+    # the hop order of the walk respects every dependency here too
+    x = B.bcast_plan_xfers(plan)
+    for chunk in range(B.bcast_plan_num_chunks(plan)):
+        for mode in (B.BCAST_EXEC_WALK, B.BCAST_EXEC_WALK_PLAN_ORDER):
+            order = B.bcast_plan_walk_order(plan, chunk, mode)
+            pos = {int(m): i for i, m in enumerate(order)}
+            for m in order:
+                d = int(x["dep"][m])
+                if d >= 0 and d in pos:
+                    assert pos[d] < pos[int(m)]
+
+
+def test_node_aware_plan_argument_errors():
+    for args in [(8, 0, 100, B.BCAST_TUNED, 0), (8, 0, 100, B.BCAST_DOUBLING, 2), (8, 9, 100, B.BCAST_TUNED, 2), (0, 0, 1, 0, 1)]:
+        with pytest.raises(B.BcastError):
+            B.bcast_plan_smp(*args)
