@@ -322,9 +322,9 @@ def run_ours(args):
     # L2 on what an earlier hop stored, so that figure is not bounded by HBM.)
     per = sorted(tuned["per"])
     launches = max(1, tuned["launches"])
-    launch_ms = statistics.mean(per) / launches
+    launch_ms = statistics.mean(per) / launches          # modes with one launch per plan step: the average launch
     floor_bytes = P * n
-    achieved = floor_bytes / (launch_ms * 1e-3) / 1e9
+    achieved = floor_bytes / launches / (launch_ms * 1e-3) / 1e9
     traffic = ncu_traffic(args.workload, args.mode)
     clocks = tuned["clocks"] or {}
     mhz, max_mhz = clocks.get("sm_mhz"), clocks.get("sm_max_mhz")
@@ -348,8 +348,8 @@ def run_ours(args):
         # every scheduled byte loaded once and stored once by the SMs (mostly L2 hits on the load side)
         "l2_level_achieved": round(2 * tuned["moved"] / launches / (launch_ms * 1e-3) / 1e9, 1),
         # the same launch counted in the DRAM bytes ncu saw (null while `traffic` is null)
-        "dram_achieved": None if traffic is None else round(traffic / (launch_ms * 1e-3) / 1e9, 1),
-        "dram_frac": None if traffic is None else round(traffic / (launch_ms * 1e-3) / 1e9 / peak, 4),
+        "dram_achieved": None if traffic is None else round(traffic / launches / (launch_ms * 1e-3) / 1e9, 1),
+        "dram_frac": None if traffic is None else round(traffic / launches / (launch_ms * 1e-3) / 1e9 / peak, 4),
     }
 
     # ---- end to end through the host-buffer entry point: H2D of the message, broadcast, D2H of all P buffers

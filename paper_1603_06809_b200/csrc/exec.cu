@@ -208,7 +208,7 @@ int walk_blocks_per_sm(int u, int P, int *bps)
 //     list at memory latency; take the smallest U whose slices fit the resident warps (the most
 //     warps, the fewest words each).
 //   * Very few ranks (P <= 4): at most three hops per slice, close to a plain copy: as many
-//     bytes in flight as the SMs hold (U = 4 for P <= 3, U = 2 for P = 4, all resident blocks).
+//     bytes in flight as the SMs hold (U = 6 for P <= 3, U = 2 for P = 4, all resident blocks).
 // BCAST_WALK_WORDS and BCAST_WALK_BLOCKS_PER_SM override the choice (for experiments).
 struct WalkShape {
     int u = 1, grid = 1;
@@ -225,7 +225,7 @@ int choose_shape(bool few_hops, const std::function<long long(int)> &slices_for,
         if ((rc = walk_blocks_per_sm(u, P, &resident))) return rc;
         bps = forced_bps > 0 ? std::min(forced_bps, resident) : resident;
     } else if (few_hops) {
-        u = P <= 3 ? 4 : 2;
+        u = P <= 3 ? 6 : 2;
         if ((rc = walk_blocks_per_sm(u, P, &resident))) return rc;
         bps = resident;
     } else if (slices_for(kMaxWords) * 5 > (long long)sm_count * kWarpsPerBlock * 7) {   // > 1.4 rounds
