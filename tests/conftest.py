@@ -15,10 +15,6 @@ def pytest_configure(config):
     ensure_built()
 
 
-def golden_path(name: str) -> str:
-    return os.path.join(ROOT, "tests", "golden", name)
-
-
 @pytest.fixture(scope="session")
 def oracle():
     from oracle import bcast_oracle
