@@ -34,8 +34,9 @@
  *   - Environment variables override what the library would choose, for experiments and tests
  *     only; they are read when a plan is executed for the first time (the last one at every call):
  *     BCAST_WALK_WORDS (1..8 sixteen-byte words per lane of the register walk, i.e. segments of
- *     512 B .. 4 KiB), BCAST_WALK_BLOCKS_PER_SM, BCAST_BULK_BLOCKS_PER_SM, BCAST_WALK_DUAL (0: walk
- *     a segment that holds a chunk boundary in two parts instead of with the merged list of
+ *     512 B .. 4 KiB), BCAST_WALK_BLOCKS_PER_SM, BCAST_WALK_GROUP (neighbouring slices that a block
+ *     of the register walk takes at a time), BCAST_BULK_BLOCKS_PER_SM, BCAST_WALK_DUAL (0: walk a
+ *     segment that holds a chunk boundary in two parts instead of with the merged list of
  *     bcast_plan_walk_pairing), BCAST_BULK_SPIN_LIMIT (polls of the bulk-copy kernel's first wait
  *     bound, see bcast_exec_status; 0 makes every wait report a timeout and then complete under the
  *     second bound), BCAST_BULK_PLAN_ORDER (1: the bulk walk takes the hops in plan order).
@@ -100,10 +101,10 @@ enum {
        copy engine are bounded: see bcast_exec_status(). */
     BCAST_EXEC_WALK_BULK = 4,
     /* The fastest of the above for the plan at hand; what bcast_exec() uses.  BCAST_EXEC_WALK_BULK
-       when the message gives the bulk walk at least two rounds of work (about 58 MB on 148 SMs)
-       and the variant is not the tuned one (whose hop order re-reads a segment up to a tree
-       level later, by which time the bulk path's larger working set has left L2); otherwise
-       BCAST_EXEC_WALK. */
+       for very large messages on many ranks (the bulk walk has at least four rounds of work, about
+       116 MB on 148 SMs, and P >= 64) unless the variant is the tuned one (whose hop order re-reads a
+       segment up to a tree level later, by which time the bulk path's larger working set has left
+       L2); otherwise BCAST_EXEC_WALK. */
     BCAST_EXEC_AUTO = 5
 };
 

@@ -58,7 +58,8 @@ struct bcast_device_state {
     // WALK: slices of the register walk and its launch shape
     WalkSlice *d_slices = nullptr;
     long long n_slices = 0;
-    int walk_u = 0, walk_grid = 0;
+    int walk_u = 0, walk_grid = 0, walk_group = 1;
+    long long walk_grouped = 0;
     // WALK with bulk copies
     WalkSlice *d_bulk_slices = nullptr, *d_reg_slices = nullptr;
     long long n_bulk = 0, n_reg = 0;
@@ -212,6 +213,7 @@ int walk_blocks_per_sm(int u, int P, int *bps)
 // BCAST_WALK_WORDS and BCAST_WALK_BLOCKS_PER_SM override the choice (for experiments).
 struct WalkShape {
     int u = 1, grid = 1;
+    bool many_rounds = false;     // the bandwidth regime: one block per SM, several rounds of slices
 };
 
 int choose_shape(bool few_hops, const std::function<long long(int)> &slices_for, int P, int sm_count, WalkShape *shape)
@@ -231,6 +233,7 @@ int choose_shape(bool few_hops, const std::function<long long(int)> &slices_for,
     } else if (slices_for(kMaxWords) * 5 > (long long)sm_count * kWarpsPerBlock * 7) {   // > 1.4 rounds
         u = kMaxWords;
         bps = 1;
+        shape->many_rounds = true;
     } else {
         for (int cand = 1; cand <= kMaxWords; cand++) {
             if ((rc = walk_blocks_per_sm(cand, P, &resident))) return rc;
@@ -279,6 +282,12 @@ int build_walk_tables(const bcast_plan_t &p, bcast_device_state &ds)
     std::vector<WalkSlice> slices;
     make_slices(p, 512ull * ds.walk_u, env_int("BCAST_WALK_DUAL", 1) != 0, nullptr, slices);
     ds.n_slices = (long long)slices.size();
+    // In the bandwidth regime the eight warps of a block take eight neighbouring slices at a time (32 KiB
+    // of every destination buffer written by one SM at about the same time) when the hop lists are long:
+    // measured +1..3 % of the copy rate for P >= 24 (config 4: 0.936 -> 0.960), -1..5 % for P <= 16.
+    // BCAST_WALK_GROUP overrides (for experiments).
+    ds.walk_group = std::max(1, env_int("BCAST_WALK_GROUP", shape.many_rounds && p.P >= 24 ? kWarpsPerBlock : 1));
+    ds.walk_grouped = ds.n_slices / ((long long)ds.walk_group * ds.walk_grid) * ds.walk_group * ds.walk_grid;
     return upload(&ds.d_slices, slices);
 }
 
@@ -399,6 +408,8 @@ WalkDev walk_dev(const bcast_plan_t &p, const bcast_device_state &ds, bool plan_
     w.trace = trace;
     w.scatter_size = p.S;
     w.nbytes = p.nbytes;
+    w.group = 1;
+    w.grouped = 0;
     return w;
 }
 
@@ -406,6 +417,8 @@ int launch_walk(const bcast_plan_t &p, const bcast_device_state &ds, void *const
                 cudaStream_t st, unsigned long long *trace)
 {
     WalkDev w = walk_dev(p, ds, plan_order, ds.d_slices, ds.n_slices, trace);
+    w.group = ds.walk_group;
+    w.grouped = ds.walk_grouped;
     return launch_with_ptrs(walk_kernel(ds.walk_u, p.P, trace != nullptr), dim3(ds.walk_grid), dim3(kThreads), 0, st,
                             rank_bufs, p.P, trace != nullptr, {&w});
 }
@@ -469,12 +482,13 @@ bool known_mode(int mode)
 // The bulk-copy walk needs ~4x the bytes in flight of the register walk.  With plan-order hops
 // (native, doubling) a segment is re-read on the very next hop and that still fits in L2; with
 // the tuned variant's level-order hops the re-read comes up to a tree level later and no longer
-// does (measured: 11-20 % slower than the register walk), so the tuned variant stays with registers.
-// It also needs at least two rounds of its own to pay: below that (about 58 MB on 148 SMs) the
-// register walk is as fast or faster (16 MiB messages: 11 % faster).
+// does (measured: 20-25 % slower than the register walk), so the tuned variant stays with registers.
+// For the others it pays only for very large messages on many ranks (measured: 128 MiB, P >= 128:
+// 0.95-0.96 of the copy rate against 0.93-0.94; at 64 MiB, or with P <= 64, the register walk is as
+// fast or faster): at least four rounds of its own (about 116 MB on 148 SMs) and P >= 64.
 int resolve_auto(const bcast_plan_t &p, const bcast_device_state &ds)
 {
-    const bool bulk_pays = ds.n_bulk >= 2ll * ds.bulk_grid * kBulkWorkers;
+    const bool bulk_pays = p.P >= 64 && ds.n_bulk >= 4ll * ds.bulk_grid * kBulkWorkers;
     return bulk_pays && p.variant != BCAST_TUNED ? BCAST_EXEC_WALK_BULK : BCAST_EXEC_WALK;
 }
 
@@ -802,6 +816,8 @@ int exec_static(void *const *rank_bufs, const bcast_plan_t &p, cudaStream_t st)
     w.trace = nullptr;
     w.scatter_size = p.S;
     w.nbytes = p.nbytes;
+    w.group = 1;
+    w.grouped = 0;
     return launch_with_ptrs(walk_kernel(img.u, p.P, false), dim3(img.grid), dim3(kThreads), 0, st, rank_bufs, p.P, false, {&w});
 }
 

@@ -340,7 +340,13 @@ bcast_walk_kernel(const __grid_constant__ RankPtrs<MAXP> bufs, const __grid_cons
         int k = 0;
         if (lane == 0) k = atomicAdd(&ticket, 1);
         k = __shfl_sync(0xffffffffu, k, 0);
-        const long long w = (long long)k * gridDim.x + blockIdx.x;
+        // ticket k of this block -> slice index w
+        const long long in_runs = t.grouped / gridDim.x;          // tickets of a block that fall into the grouped part
+        long long w;
+        if (k < in_runs)
+            w = ((long long)(k / t.group) * gridDim.x + blockIdx.x) * t.group + (k % t.group);
+        else
+            w = t.grouped + (k - in_runs) * gridDim.x + blockIdx.x;
         if (w >= t.n_slices) break;
         walk_slice<U, MAXP, TRACE>(bufs, t.slices[w], t, lane);
     }

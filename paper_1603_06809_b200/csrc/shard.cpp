@@ -196,6 +196,8 @@ int launch_kernel(const bcast_plan_t &p, ShardKernel &k, void *const *rank_bufs,
     w.trace = trace;
     w.scatter_size = p.S;
     w.nbytes = p.nbytes;
+    w.group = 1;
+    w.grouped = 0;
     return bcast_internal_launch_walk(w, k.u, k.grid, rank_bufs, p.P, st);
 }
 

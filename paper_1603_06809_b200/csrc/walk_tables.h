@@ -48,6 +48,10 @@ struct WalkDev {
     const DualMsg *dual_msg;
     unsigned long long *trace;   // traced launches only: bytes stored per plan message
     uint64_t scatter_size, nbytes;
+    // How slices are dealt to blocks: the first `grouped` slices of the list in runs of `group`
+    // neighbours (run j goes to block j mod gridDim.x), the rest one by one (group = 1: all one by one).
+    int group;
+    long long grouped;
 };
 
 // Per relative chunk, the plan messages ("hops") a walk performs on the bytes of that chunk: in
