@@ -696,7 +696,8 @@ struct bcast_static_image {
     std::vector<unsigned char> bytes;
     size_t off_dual_begin = 0, off_slices = 0, off_hops = 0, off_dual = 0;
     long long n_slices = 0;
-    int u = 0, grid = 0, sm_count = 0;
+    int u = 0, grid = 0, sm_count = 0, group = 1;
+    long long grouped = 0;
 };
 
 void bcast_static_image_free(bcast_static_image *img) { delete img; }
@@ -760,6 +761,8 @@ int make_static_image(const bcast_plan_t &p, int sm_count, bcast_static_image &i
         img.n_slices = (long long)slices.size();
         img.u = u;
         img.grid = (int)std::max<long long>(1, std::min<long long>(shape.grid, img.n_slices));
+        img.group = shape.many_rounds && u == shape.u && p.P >= 24 ? kWarpsPerBlock : 1;     // as in build_walk_tables
+        img.grouped = img.n_slices / ((long long)img.group * img.grid) * img.group * img.grid;
         img.sm_count = sm_count;
         return BCAST_OK;
     }
@@ -816,8 +819,8 @@ int exec_static(void *const *rank_bufs, const bcast_plan_t &p, cudaStream_t st)
     w.trace = nullptr;
     w.scatter_size = p.S;
     w.nbytes = p.nbytes;
-    w.group = 1;
-    w.grouped = 0;
+    w.group = img.group;
+    w.grouped = img.grouped;
     return launch_with_ptrs(walk_kernel(img.u, p.P, false), dim3(img.grid), dim3(kThreads), 0, st, rank_bufs, p.P, false, {&w});
 }
 
