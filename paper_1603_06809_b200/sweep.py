@@ -5,7 +5,8 @@
 
 For every workload: median time of the tuned and of the native variant (and, where P is a power of
 two, of the scatter + recursive-doubling variant) (CUDA events around each
-execution, after warm-up), the effective broadcast rate P*nbytes/t, the algorithmic rate
+execution, after warm-up), the effective broadcast rate P*nbytes/t and its fraction of the measured
+plain-copy rate (P*nbytes is what a broadcast cannot avoid moving through DRAM), the L2-level rate
 2*sum(len)/t, and the tuned-over-native speed-up.  After timing, every rank buffer is compared with
 the root's message on the device.  Uses only the CUDA library: no CPU path is involved.
 """
@@ -13,6 +14,7 @@ from __future__ import annotations
 
 import argparse
 import json
+import os
 import statistics
 
 import torch
@@ -51,7 +53,19 @@ def time_workload(wl: W.Workload, variant: int, mode: int, iters: int, warmup: i
     return ms, B.bcast_plan_total_bytes(plan)
 
 
+def copy_rate_gbs() -> float:
+    """The measured plain-copy rate of this machine's GPUs (MEASURED_PEAKS.json at the repository root),
+    else the nominal 8000 GB/s: the denominator of the roofline fraction."""
+    path = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"])
+    except Exception:
+        return 8000.0
+
+
 def run(workloads, mode: int, iters: int):
+    peak = copy_rate_gbs()
     rows = []
     for wl in workloads:
         it = iters if wl.total_bytes < (1 << 30) else max(5, iters // 5)
@@ -65,6 +79,9 @@ def run(workloads, mode: int, iters: int):
             "doubling_us": None if d_ms is None else round(d_ms * 1e3, 2),
             "tuned_us": round(t_ms * 1e3, 2), "native_us": round(n_ms * 1e3, 2),
             "tuned_effective_GBps": round(wl.P * wl.nbytes / t_ms / 1e6, 1),
+            # DRAM floor of a broadcast (message read once, every other buffer written once = P*nbytes) over the copy rate
+            "tuned_roofline_frac": round(wl.P * wl.nbytes / t_ms / 1e6 / peak, 4),
+            "native_roofline_frac": round(wl.P * wl.nbytes / n_ms / 1e6 / peak, 4),
             "tuned_algorithmic_GBps": round(2 * t_bytes / t_ms / 1e6, 1),
             "native_algorithmic_GBps": round(2 * n_bytes / n_ms / 1e6, 1),
             "bytes_native_over_tuned": round(n_bytes / t_bytes, 4) if t_bytes else None,
@@ -90,11 +107,11 @@ def main():
         for r in rows:
             print(json.dumps(r))
         return
-    print(f"{'workload':28s} {'tuned us':>10s} {'native us':>10s} {'P*n/t GB/s':>11s} {'alg GB/s':>10s} "
+    print(f"{'workload':28s} {'tuned us':>10s} {'native us':>10s} {'P*n/t GB/s':>11s} {'roofline':>8s} {'L2 GB/s':>10s} "
           f"{'bytes n/t':>9s} {'speed-up':>8s} {'doubling us':>11s}")
     for r in rows:
         print(f"{r['workload']:28s} {r['tuned_us']:10.2f} {r['native_us']:10.2f} {r['tuned_effective_GBps']:11.1f} "
-              f"{r['tuned_algorithmic_GBps']:10.1f} {r['bytes_native_over_tuned']:9.4f} {r['speedup_tuned_over_native']:8.4f} "
+              f"{r['tuned_roofline_frac']:8.3f} {r['tuned_algorithmic_GBps']:10.1f} {r['bytes_native_over_tuned']:9.4f} {r['speedup_tuned_over_native']:8.4f} "
               f"{'' if r['doubling_us'] is None else format(r['doubling_us'], '11.2f')}")
 
 
