@@ -323,11 +323,14 @@ __device__ __forceinline__ void walk_slice(const RankPtrs<MAXP> &bufs, const Wal
     else walk_ragged<U, MAXP, TRACE>(bufs, sl.seg, c, t, lane);
 }
 
-// Slices are dealt round-robin over the blocks (slice w belongs to block w mod gridDim.x), so that
-// every SM gets the same share and the slices in flight at any time are neighbours in the message;
-// inside a block the warps draw the block's slices in order from a ticket counter in shared
-// memory, so a warp that got a slow slice (a partial sector at the end of the message, an L2 miss)
-// does not hold up the others.  Warps never wait for one another.
+// Slices are dealt round-robin over the blocks -- one by one (slice w belongs to block
+// w mod gridDim.x) or, for the first `grouped` slices of the list, in runs of `group` neighbours
+// (run j belongs to block j mod gridDim.x; with group = warps per block an SM then works on one
+// contiguous piece of the message at a time) -- so that every SM gets the same share and the
+// slices in flight at any time are neighbours in the message.  Inside a block the warps draw the
+// block's slices in order from a ticket counter in shared memory, so a warp that got a slow
+// slice (a partial sector at the end of the message, an L2 miss) does not hold up the others.
+// Warps never wait for one another.
 template <int U, int MAXP, bool TRACE>
 __global__ void __launch_bounds__(kThreads)
 bcast_walk_kernel(const __grid_constant__ RankPtrs<MAXP> bufs, const __grid_constant__ WalkDev t)
