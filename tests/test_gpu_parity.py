@@ -336,3 +336,51 @@ def test_node_aware_broadcast(oracle, wl, c, variant, mode):
         torch.cuda.synchronize()
         assert np.array_equal(counts.cpu().numpy(), ref.col("len"))       # every message performed in full, once
         assert bufs.all_equal_message()
+
+
+# ---- seeded random shapes: every kind of slice (whole, cut by one boundary, cut by several, message
+# tail), every variant, the executors in turn
+def _random_cases(count, seed):
+    rng = np.random.default_rng(seed)
+    cases = []
+    for i in range(count):
+        P = int(rng.choice([2, 3, 5, 9, 17, 31, 48, 64, 100, 129, 200, 255, 300]))
+        kind = i % 4
+        if kind == 0:
+            n = int(rng.integers(1, 4 * P))                      # chunks of a few bytes, some empty
+        elif kind == 1:
+            n = int(rng.integers(P * 40, P * 700))               # several boundaries per 512-byte segment
+        elif kind == 2:
+            n = int(rng.integers(P * 3000, P * 9000))            # one boundary per segment at most
+        else:
+            n = int(rng.integers(1 << 20, 3 << 20))              # a megabyte or so, odd
+        cases.append((P, int(rng.integers(0, P)), n, int(rng.integers(0, 3)), i))
+    return cases
+
+
+@pytest.mark.parametrize("P,root,n,variant,i", _random_cases(48, 20261130))
+def test_random_shapes(oracle, P, root, n, variant, i):
+    if variant == B.BCAST_DOUBLING and P & (P - 1):
+        variant = B.BCAST_TUNED
+    mode = MODES[i % len(MODES)]
+    check_against_oracle(oracle, W.Workload(f"random_{i}", P, root, n, 900 + i), variant, mode, shift=16 * (i % 2))
+    # and the same shape node-aware, or spread over a partition, with the bytes counted on the device
+    msg = W.message_bytes(900 + i, n)
+    if variant != B.BCAST_DOUBLING and i % 3 == 0:
+        c = int(1 + (i * 7) % max(1, P // 2))
+        plan, bufs = run_broadcast(P, root, n, variant, mode, msg, ranks_per_node=c)
+        ref = oracle.simulate(P, root, n, variant, message=msg, ranks_per_node=c)
+        assert np.array_equal(bufs.to_host(), ref.bufs) and bufs.guards_intact()
+    if i % 3 == 1:
+        G = int(min(P, 2 + i % 5))
+        bufs = RankBuffers(P, root, n, msg)
+        plan = B.bcast_plan(P, root, n, variant)
+        shard = B.bcast_shard_create(plan, G)
+        counts = torch.zeros(max(1, B.bcast_plan_num_xfers(plan)), dtype=torch.int64, device="cuda:0")
+        st = torch.cuda.current_stream()
+        torch.cuda.synchronize()
+        B.bcast_shard_exec(shard, bufs.pointers(), [0] * G, [st] * G, counts)
+        torch.cuda.synchronize()
+        ref = oracle.simulate(P, root, n, variant, message=msg)
+        assert np.array_equal(bufs.to_host(), ref.bufs) and bufs.guards_intact()
+        assert np.array_equal(counts.cpu().numpy()[: len(ref.schedule)], ref.col("len"))
