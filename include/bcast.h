@@ -387,8 +387,9 @@ int64_t bcast_shard_hops(const bcast_shard_t *shard, int phase, int gpu, int chu
 /*
  * bcast_shard_exec -- perform the whole plan from one process that drives all GPUs.
  *   rank_bufs     HOST array of P DEVICE pointers; rank r's buffer must be memory of device
- *                 gpu_device[rank_gpu[r]] (peer access between those devices enabled by the caller
- *                 where they differ); alignment and disjointness as for bcast_exec
+ *                 gpu_device[rank_gpu[r]]; alignment and disjointness as for bcast_exec.  Where the
+ *                 devices differ the first call enables peer access between them (BCAST_ERR_INVAL if
+ *                 two of them cannot reach each other)
  *   gpu_device    HOST array [num_gpus]: CUDA device ordinal of every GPU of the partition (they may
  *                 repeat: several, or all, "GPUs" of the partition on one device); fixed by the first call
  *   cuda_streams  HOST array [num_gpus] of cudaStream_t, stream g on device gpu_device[g]; streams of

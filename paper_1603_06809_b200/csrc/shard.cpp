@@ -216,9 +216,33 @@ int check_placement(const bcast_shard &sh, void *const *rank_bufs, const int *de
     return BCAST_OK;
 }
 
+// Every device of the partition must be able to load from every other one's memory: enable peer
+// access where it is not enabled yet (one process driving all GPUs; with one process per GPU the
+// IPC mappings the caller opens do this).
+int enable_peer_access(const int *devices, int G)
+{
+    int cur = -1;
+    SHARD_TRY(cudaGetDevice(&cur));
+    for (int a = 0; a < G; a++)
+        for (int b = 0; b < G; b++) {
+            if (devices[a] == devices[b]) continue;
+            int can = 0;
+            SHARD_TRY(cudaDeviceCanAccessPeer(&can, devices[a], devices[b]));
+            if (!can) { cudaSetDevice(cur); return BCAST_ERR_INVAL; }
+            SHARD_TRY(cudaSetDevice(devices[a]));
+            const cudaError_t e = cudaDeviceEnablePeerAccess(devices[b], 0);
+            if (e == cudaErrorPeerAccessAlreadyEnabled) cudaGetLastError();      // fine: clear it
+            else if (e != cudaSuccess) { cudaSetDevice(cur); return bcast_internal_cuda_failed((int)e); }
+        }
+    SHARD_TRY(cudaSetDevice(cur));
+    return BCAST_OK;
+}
+
 int fix_devices(bcast_shard &sh, const int *devices)
 {
     if (sh.devices.empty()) {
+        const int rc = enable_peer_access(devices, sh.G);
+        if (rc) return rc;
         sh.devices.assign(devices, devices + sh.G);
         return BCAST_OK;
     }
