@@ -115,11 +115,11 @@ def test_runs_on_a_side_stream(oracle):
 def test_cfg4_full_size(oracle, variant):
     wl = W.CFG4
     msg = W.message_bytes(wl.seed, wl.nbytes)
-    for mode in (B.BCAST_EXEC_WALK, B.BCAST_EXEC_AUTO):         # AUTO is the bulk-copy kernel at this size
+    for mode in (B.BCAST_EXEC_WALK_BULK, B.BCAST_EXEC_AUTO):    # AUTO (what bench.py times) is the register walk at this size
         plan, bufs = run_broadcast(wl.P, wl.root, wl.nbytes, variant, mode, msg)
         assert bufs.all_equal_message() and bufs.guards_intact()
         B.bcast_exec_status(plan)
-        if mode == B.BCAST_EXEC_WALK:
+        if mode == B.BCAST_EXEC_WALK_BULK:
             del bufs
             torch.cuda.empty_cache()
     ref = oracle.simulate(wl.P, wl.root, wl.nbytes, variant, message=msg)
