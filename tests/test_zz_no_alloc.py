@@ -125,3 +125,14 @@ def test_static_refuses_a_capturing_stream():
     B.bcast_exec_static(bufs.pointers(), plan, torch.cuda.current_stream())   # still usable afterwards
     torch.cuda.synchronize()
     assert bufs.all_equal_message() and bufs.guards_intact()
+
+
+def test_static_falls_back_when_the_boundary_lists_do_not_fit():
+    # P = 512 with an odd scatter size: hop lists (4 P^2 bytes) fit into the built-in array, the merged
+    # boundary lists on top of them do not; the call then walks cut segments in two parts instead
+    wl = W.Workload("static_p512", 512, 77, 512 * 2051 + 9, 45)
+    msg = W.message_bytes(wl.seed, wl.nbytes)
+    got = run(B.bcast_exec_static, wl, B.BCAST_TUNED, msg)
+    assert (got == msg[None, :]).all()
+    want = run(B.bcast_exec, wl, B.BCAST_TUNED, msg)
+    assert np.array_equal(got, want)
