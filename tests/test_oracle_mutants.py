@@ -83,6 +83,8 @@ def schedule_level_pins(oracle):
     for case in pins.SMP_CASES:
         yield lambda case=case: pins.test_node_aware_structure(oracle, *case)
     yield lambda: pins.test_node_aware_degenerate_cases(oracle)
+    for case in pins.SMP_CASES[:3]:
+        yield lambda case=case: pins.test_node_aware_dep_names_the_last_writer(oracle, *case)
     yield lambda: pins.test_node_aware_leader_ring_is_the_plain_ring_of_the_nodes(oracle)
 
 

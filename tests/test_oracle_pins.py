@@ -560,3 +560,28 @@ def test_node_aware_degenerate_cases(oracle):
         assert {(int(r[1]), int(r[2]), int(r[3])) for r in one.schedule} == tree_by_halving(members)
     with pytest.raises(oracle.OracleError):
         oracle.simulate(8, 0, 100, 2, ranks_per_node=2)              # no recursive doubling between nodes here
+
+
+@pytest.mark.parametrize("P,root,n,c", SMP_CASES)
+def test_node_aware_dep_names_the_last_writer(oracle, P, root, n, c):
+    """`dep` of every message of the node-aware schedule is the message that last wrote the first chunk
+    it carries into its source (-1: the root's own data), and lies in an earlier step; messages of one
+    step are listed by destination."""
+    k = -(-P // c)
+    for variant in (NATIVE, TUNED):
+        sched = oracle.simulate(P, root, n, variant, ranks_per_node=c).schedule
+        holds = {(root, cc): -1 for cc in range(k)}
+        i = 0
+        while i < len(sched):
+            j = i
+            while j < len(sched) and (sched[j, 0], sched[j, 1]) == (sched[i, 0], sched[i, 1]):
+                j += 1
+            assert list(sched[i:j, 3]) == sorted(sched[i:j, 3]) and len(set(sched[i:j, 3])) == j - i
+            for x in range(i, j):
+                src, first, dep = int(sched[x, 2]), int(sched[x, 4]), int(sched[x, 8])
+                assert dep == holds[(src, first)] and dep < i
+            for x in range(i, j):
+                for cc in range(int(sched[x, 4]), int(sched[x, 4] + sched[x, 5])):
+                    holds[(int(sched[x, 3]), cc)] = x
+            i = j
+        assert len(holds) == P * k
