@@ -253,6 +253,15 @@ int choose_shape(bool few_hops, const std::function<long long(int)> &slices_for,
     return BCAST_OK;
 }
 
+// In the bandwidth regime the eight warps of a block take eight neighbouring slices at a time (32 KiB
+// of every destination buffer written by one SM at about the same time) when the hop lists are long:
+// measured +1..3 % of the copy rate for P >= 24 (config 4: 0.936 -> 0.960), -1..5 % for P <= 16.
+// BCAST_WALK_GROUP overrides (for experiments).
+int walk_group_for(const WalkShape &shape, int P)
+{
+    return std::max(1, env_int("BCAST_WALK_GROUP", shape.many_rounds && P >= 24 ? kWarpsPerBlock : 1));
+}
+
 int choose_walk_shape(const bcast_plan_t &p, int sm_count, WalkShape *shape)
 {
     return choose_shape(p.P <= 4, [&](int u) { return count_slices(p, 512ull * u, true, nullptr); }, p.P, sm_count, shape);
@@ -282,11 +291,7 @@ int build_walk_tables(const bcast_plan_t &p, bcast_device_state &ds)
     std::vector<WalkSlice> slices;
     make_slices(p, 512ull * ds.walk_u, env_int("BCAST_WALK_DUAL", 1) != 0, nullptr, slices);
     ds.n_slices = (long long)slices.size();
-    // In the bandwidth regime the eight warps of a block take eight neighbouring slices at a time (32 KiB
-    // of every destination buffer written by one SM at about the same time) when the hop lists are long:
-    // measured +1..3 % of the copy rate for P >= 24 (config 4: 0.936 -> 0.960), -1..5 % for P <= 16.
-    // BCAST_WALK_GROUP overrides (for experiments).
-    ds.walk_group = std::max(1, env_int("BCAST_WALK_GROUP", shape.many_rounds && p.P >= 24 ? kWarpsPerBlock : 1));
+    ds.walk_group = walk_group_for(shape, p.P);
     ds.walk_grouped = ds.n_slices / ((long long)ds.walk_group * ds.walk_grid) * ds.walk_group * ds.walk_grid;
     return upload(&ds.d_slices, slices);
 }
@@ -522,12 +527,13 @@ int exec_checked(void *const *rank_bufs, const bcast_plan_t *plan, void *cuda_st
 
 // ======================================================================================= for shard.cpp
 int bcast_internal_walk_shape(bool few_hops, const std::function<long long(int)> &slices_for, int P, int sm_count, int *u,
-                              int *grid)
+                              int *grid, int *group)
 {
     WalkShape shape;
     const int rc = choose_shape(few_hops, slices_for, P, sm_count, &shape);
     *u = shape.u;
     *grid = shape.grid;
+    *group = walk_group_for(shape, P);
     return rc;
 }
 
@@ -761,7 +767,7 @@ int make_static_image(const bcast_plan_t &p, int sm_count, bcast_static_image &i
         img.n_slices = (long long)slices.size();
         img.u = u;
         img.grid = (int)std::max<long long>(1, std::min<long long>(shape.grid, img.n_slices));
-        img.group = shape.many_rounds && u == shape.u && p.P >= 24 ? kWarpsPerBlock : 1;     // as in build_walk_tables
+        img.group = u == shape.u ? walk_group_for(shape, p.P) : 1;                            // as in build_walk_tables
         img.grouped = img.n_slices / ((long long)img.group * img.grid) * img.group * img.grid;
         img.sm_count = sm_count;
         return BCAST_OK;

@@ -6,8 +6,9 @@
 
 // Launch shape of a register walk: words per lane (1..8) and blocks, for a walk whose slice count
 // at `u` words per lane is slices_for(u).  `few_hops`: the longest hop list has at most three hops.
+// *group: how many neighbouring slices a block takes at a time (WalkDev::group).
 int bcast_internal_walk_shape(bool few_hops, const std::function<long long(int)> &slices_for, int P, int sm_count, int *u,
-                              int *grid);
+                              int *grid, int *group);
 
 // Enqueue one register-walk kernel (traced if w.trace is set) on the current device.
 int bcast_internal_launch_walk(const WalkDev &w, int u, int grid, void *const *rank_bufs, int P, void *cuda_stream);

@@ -43,8 +43,8 @@ struct ShardKernel {               // one (phase, gpu) launch
     bool any = false;
     // device side (on the GPU's device), built at the first execution
     bool built = false;
-    int u = 0, grid = 0;
-    long long n_slices = 0;
+    int u = 0, grid = 0, group = 1;
+    long long n_slices = 0, grouped = 0;
     WalkSlice *d_slices = nullptr;
     uint32_t *d_hops = nullptr;
     int32_t *d_hop_msg = nullptr;
@@ -161,11 +161,12 @@ int build_kernel(const bcast_plan_t &p, ShardKernel &k)
     WalkTables t;
     make_walk_tables(p, k.lists, t);
     int rc = bcast_internal_walk_shape(false, [&](int u) { return count_slices(p, 512ull * u, true, &k.active); }, p.P, sms,
-                                       &k.u, &k.grid);
+                                       &k.u, &k.grid, &k.group);
     if (rc) return rc;
     std::vector<WalkSlice> slices;
     make_slices(p, 512ull * k.u, true, &k.active, slices);
     k.n_slices = (long long)slices.size();
+    k.grouped = k.n_slices / ((long long)k.group * k.grid) * k.group * k.grid;
     if ((rc = upload(&k.d_slices, slices))) return rc;
     if ((rc = upload(&k.d_hops, t.hops))) return rc;
     if ((rc = upload(&k.d_hop_msg, t.hop_msg))) return rc;
@@ -196,8 +197,8 @@ int launch_kernel(const bcast_plan_t &p, ShardKernel &k, void *const *rank_bufs,
     w.trace = trace;
     w.scatter_size = p.S;
     w.nbytes = p.nbytes;
-    w.group = 1;
-    w.grouped = 0;
+    w.group = k.group;
+    w.grouped = k.grouped;
     return bcast_internal_launch_walk(w, k.u, k.grid, rank_bufs, p.P, st);
 }
 
